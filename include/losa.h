@@ -1,0 +1,143 @@
+/*
+ * liblosa — LoSA's attention hot path for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * LoSA ("Near-Lossless Sparse Attention", Methodology section) measures the
+ * exact block attention mass of one dense attention step, keeps for every
+ * (head, query block) the smallest set of key/value blocks whose mass reaches
+ * a threshold tau, and reuses those frozen block indices in a block-sparse
+ * attention forward at every later step.  This library is that path:
+ *
+ *     losa_block_mass   Eq. 1   q, k            -> mass[B, H, nQb, nKb]
+ *     losa_select       Eq. 3   mass, tau       -> CSR (offsets, kv_idx)
+ *     losa_sparse_attn  Eq. 4   q, k, v, CSR    -> o
+ *     losa_attn         dense softmax attention (the warm-up steps and the
+ *                       denominator of the sparse-versus-dense ratio)
+ *
+ * Conventions shared by every call
+ * --------------------------------
+ *  - All tensor pointers are DEVICE pointers on the current CUDA device,
+ *    16-byte aligned.  The caller owns every buffer, including workspace;
+ *    the library allocates no device memory per call (it keeps one small
+ *    pinned status word and cached device properties per process).
+ *  - q, k, v, o are [B, H, N, D] with element strides (sb, sh, sn) and D
+ *    contiguous; strides must be multiples of 8 elements.  q, k, v are bf16.
+ *    N is the number of VALID tokens and need not be a multiple of the block
+ *    sizes: the last query/key block is short, tokens >= N do not exist (they
+ *    enter no softmax and no mass) and rows >= N of o are never written.
+ *  - nQb = ceil(N / R), nKb = ceil(N / C).  A "row" is one (b, h, i) query
+ *    block, numbered (b*H + h)*nQb + i.
+ *  - Calls enqueue work on `cuda_stream` (a cudaStream_t; NULL = default
+ *    stream) and return without synchronising.  The return value reports
+ *    errors found on the host before any launch.  Errors found on the device
+ *    (a bounded wait that expired, a bad block index, a negative mass, a CSR
+ *    that overflowed its capacity) are recorded in a status word that
+ *    losa_async_status() returns and clears.  No kernel ever traps, asserts
+ *    or waits without a bound.
+ *  - Supported shapes: D in {64, 128}; (R, C) in {(64, 64), (128, 128)}.
+ */
+#ifndef LOSA_H_
+#define LOSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  LOSA_OK = 0,
+  LOSA_ERR_INVALID_ARG = -1, /* null / misaligned pointer, bad size, tau outside (0, 1]      */
+  LOSA_ERR_UNSUPPORTED = -2, /* D, R, C, dtype or device not supported                       */
+  LOSA_ERR_WORKSPACE = -3,   /* workspace smaller than losa_workspace_bytes()                */
+  LOSA_ERR_CAPACITY = -4,    /* CSR longer than kv_capacity (device-side)                    */
+  LOSA_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed                            */
+  LOSA_ERR_TIMEOUT = -6,     /* a bounded device-side wait expired (device-side)             */
+  LOSA_ERR_BAD_INDEX = -7,   /* kv_idx / offsets out of range or not ascending (device-side) */
+  LOSA_ERR_BAD_MASS = -8     /* negative or NaN mass seen by losa_select (device-side)       */
+};
+
+enum { LOSA_OP_BLOCK_MASS = 0, LOSA_OP_SELECT = 1, LOSA_OP_SPARSE_ATTN = 2, LOSA_OP_ATTN = 3 };
+
+enum { LOSA_DTYPE_BF16 = 0, LOSA_DTYPE_F32 = 1 };
+
+typedef struct {
+  int32_t B, H, N, D; /* batch, heads, VALID tokens, head dimension                     */
+  int32_t R, C;       /* query / key-value block size                                   */
+  int64_t sb, sh, sn; /* element strides of batch, head, token (D is contiguous)        */
+  float scale;        /* softmax scale; 0 selects 1/sqrt(D) as in A = softmax(QK^T/sqrt d) */
+} losa_problem_t;
+
+/* Bytes of caller-provided device workspace an operation needs for this problem
+ * (LOSA_OP_*).  For LOSA_OP_SELECT only B, H, N, R, C are read.  Returns 0 for
+ * operations that need none, and 0 for an invalid problem.  Host-only: touches no GPU. */
+size_t losa_workspace_bytes(int op, const losa_problem_t* p);
+
+/* Exact block attention mass of one dense attention step (Eq. 1).
+ * For every row (b, h, i) and key block j:
+ *     mass[b,h,i,j] = (1/|B^Q_i|) * sum_{q in B^Q_i} sum_{k in B^K_j} A(q,k),
+ *     A = row-wise softmax(q k^T * scale) over the N valid keys,
+ * i.e. the paper's M(i,j) divided by the number of valid rows of query block i, so
+ * that each row of `mass` sums to 1 and Eq. 3's threshold theta*R becomes tau.
+ * The softmax is computed with a running maximum and sum; the per-key-block sums are
+ * taken in the same pass.
+ *   q, k    bf16 [B,H,N,D] (strides from p)
+ *   mass    f32  [B,H,nQb,nKb] contiguous, fully overwritten
+ *   lse     f32  [B,H,N] contiguous or NULL: natural-log sum-exp of each row's scaled scores
+ *   ws      >= losa_workspace_bytes(LOSA_OP_BLOCK_MASS, p) bytes, contents undefined after */
+int losa_block_mass(const losa_problem_t* p, const void* q, const void* k, float* mass,
+                    float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Retained-mass selection (Eq. 3).  For every row r = (b, h, i): sort the nKb masses in
+ * decreasing order (equal masses: lower block index first), accumulate them in fp64 and
+ * keep the shortest prefix whose sum is >= tau; tau >= 1 keeps every block, and so does a
+ * row whose sum never reaches tau.  Each row keeps at least one block.
+ *   mass        f32 [rows, nKb], rows = B*H*nQb, values >= 0
+ *   tau         in (0, 1]
+ *   offsets     i32 [rows + 1]: exclusive prefix of the per-row counts; offsets[rows] = nnz
+ *   kv_idx      i32 [kv_capacity]: kept block indices, row after row, ascending in a row
+ *   kv_capacity rows*nKb always suffices; if nnz exceeds it nothing past the capacity is
+ *               written and the status word becomes LOSA_ERR_CAPACITY (offsets stay exact)
+ *   ws          >= losa_workspace_bytes(LOSA_OP_SELECT, p) bytes                          */
+int losa_select(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const float* mass, double tau,
+                int32_t* offsets, int32_t* kv_idx, int64_t kv_capacity, void* ws,
+                size_t ws_bytes, void* cuda_stream);
+
+/* Block-sparse attention with a frozen pattern (Eq. 4).  Every valid query row q of query
+ * block i attends to the valid keys of the blocks kv_idx[offsets[r] .. offsets[r+1]) only;
+ * the softmax denominator runs over those keys only:
+ *     o(q) = sum_{k in K(q)} softmax_{K(q)}(q k^T * scale) v(k).
+ * The CSR must satisfy losa_validate_csr(); a block index outside [0, nKb) is skipped and
+ * reported as LOSA_ERR_BAD_INDEX, never dereferenced.
+ *   q, k, v  bf16 [B,H,N,D];  o  [B,H,N,D] with the same strides, bf16 or f32 (o_dtype)   */
+int losa_sparse_attn(const losa_problem_t* p, const void* q, const void* k, const void* v,
+                     const int32_t* offsets, const int32_t* kv_idx, void* o, int o_dtype,
+                     void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Dense softmax attention o = softmax(q k^T * scale) v over the N valid keys: the paper's
+ * dense steps up to the construction step, and this library's own dense baseline.
+ * Same tensors as losa_sparse_attn without the CSR. */
+int losa_attn(const losa_problem_t* p, const void* q, const void* k, const void* v, void* o,
+              int o_dtype, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Checks a CSR on the device: offsets[0] == 0, offsets non-decreasing with every row
+ * holding between 1 and nKb entries (Eq. 3 keeps at least one block), indices in
+ * [0, nKb) and strictly ascending inside a row.  A violation sets the status word to
+ * LOSA_ERR_BAD_INDEX.  Needs no workspace. */
+int losa_validate_csr(int32_t rows, int32_t nKb, const int32_t* offsets, const int32_t* kv_idx,
+                      void* cuda_stream);
+
+/* Synchronises `cuda_stream`, then returns and clears the device-side status word
+ * (LOSA_OK or the first device-side LOSA_ERR_* recorded since the last call). */
+int losa_async_status(void* cuda_stream);
+
+/* Static, human-readable name of a status code. */
+const char* losa_status_string(int status);
+
+/* Text of the last host-side CUDA error seen by this thread's calls ("" if none). */
+const char* losa_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOSA_H_ */

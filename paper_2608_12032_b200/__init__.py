@@ -1,0 +1,18 @@
+"""LoSA attention hot path for B200: block-mass pass, retained-mass selection, block-sparse
+attention and the library's own dense attention, as hand-written sm_100a CUDA kernels behind a
+C-ABI shared library (``liblosa.so``) with a ctypes binding of the same names."""
+from . import inputs  # noqa: F401  (seeded synthetic workloads; no method arithmetic)
+from .binding import (  # noqa: F401
+    LosaError,
+    Problem,
+    check_async,
+    losa_async_status,
+    losa_attn,
+    losa_block_mass,
+    losa_select,
+    losa_sparse_attn,
+    losa_status_string,
+    losa_validate_csr,
+    losa_workspace_bytes,
+    make_problem,
+)

@@ -1,0 +1,231 @@
+"""ctypes binding of liblosa.so: argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels.  PyTorch supplies device
+memory and the current stream.  There is no CPU fallback: if the library cannot be
+loaded the import of a function from here raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "liblosa.so")
+
+LOSA_OP_BLOCK_MASS, LOSA_OP_SELECT, LOSA_OP_SPARSE_ATTN, LOSA_OP_ATTN = 0, 1, 2, 3
+LOSA_DTYPE_BF16, LOSA_DTYPE_F32 = 0, 1
+
+EXPORTS = (
+    "losa_workspace_bytes", "losa_block_mass", "losa_select", "losa_sparse_attn", "losa_attn",
+    "losa_validate_csr", "losa_async_status", "losa_status_string", "losa_last_cuda_error",
+)
+
+
+class LosaError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        lib = _lib()
+        name = lib.losa_status_string(code).decode()
+        detail = lib.losa_last_cuda_error().decode()
+        super().__init__(f"{where}: {name}" + (f" ({detail})" if detail and code == -5 else ""))
+
+
+class Problem(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("H", ctypes.c_int32), ("N", ctypes.c_int32), ("D", ctypes.c_int32),
+        ("R", ctypes.c_int32), ("C", ctypes.c_int32),
+        ("sb", ctypes.c_int64), ("sh", ctypes.c_int64), ("sn", ctypes.c_int64),
+        ("scale", ctypes.c_float),
+    ]
+
+
+_LIB = None
+
+
+def _lib():
+    global _LIB
+    if _LIB is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2608_12032_b200.build` "
+                "(there is no fallback path)"
+            )
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+        pp = ctypes.POINTER(Problem)
+        lib.losa_workspace_bytes.restype = sz
+        lib.losa_workspace_bytes.argtypes = [ctypes.c_int, pp]
+        lib.losa_block_mass.restype = ctypes.c_int
+        lib.losa_block_mass.argtypes = [pp, vp, vp, vp, vp, vp, sz, vp]
+        lib.losa_select.restype = ctypes.c_int
+        lib.losa_select.argtypes = [i32, i32, i32, i32, vp, ctypes.c_double, vp, vp, i64, vp, sz, vp]
+        lib.losa_sparse_attn.restype = ctypes.c_int
+        lib.losa_sparse_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, ctypes.c_int, vp, sz, vp]
+        lib.losa_attn.restype = ctypes.c_int
+        lib.losa_attn.argtypes = [pp, vp, vp, vp, vp, ctypes.c_int, vp, sz, vp]
+        lib.losa_validate_csr.restype = ctypes.c_int
+        lib.losa_validate_csr.argtypes = [i32, i32, vp, vp, vp]
+        lib.losa_async_status.restype = ctypes.c_int
+        lib.losa_async_status.argtypes = [vp]
+        lib.losa_status_string.restype = ctypes.c_char_p
+        lib.losa_status_string.argtypes = [ctypes.c_int]
+        lib.losa_last_cuda_error.restype = ctypes.c_char_p
+        lib.losa_last_cuda_error.argtypes = []
+        _LIB = lib
+    return _LIB
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != 0:
+        raise LosaError(rc, where)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def make_problem(q: torch.Tensor, R: int, C: int, scale: Optional[float] = None) -> Problem:
+    if q.dim() != 4 or q.stride(3) != 1:
+        raise ValueError("expected [B, H, N, D] with a contiguous last dimension")
+    B, H, N, D = q.shape
+    return Problem(B, H, N, D, R, C, q.stride(0), q.stride(1), q.stride(2),
+                   0.0 if scale is None else float(scale))
+
+
+def _same_layout(ref: torch.Tensor, *others: torch.Tensor) -> None:
+    for t in others:
+        if t.shape != ref.shape or t.stride() != ref.stride():
+            raise ValueError("q, k, v (and o) must share shape and strides")
+        if t.device != ref.device:
+            raise ValueError("tensors must live on the same device")
+
+
+def losa_workspace_bytes(op: int, problem: Problem) -> int:
+    return int(_lib().losa_workspace_bytes(op, ctypes.byref(problem)))
+
+
+def _workspace(op: int, problem: Problem, device, ws: Optional[torch.Tensor]) -> Tuple[Optional[torch.Tensor], int]:
+    need = losa_workspace_bytes(op, problem)
+    if ws is None and need > 0:
+        ws = torch.empty(need, dtype=torch.uint8, device=device)
+    return ws, (0 if ws is None else ws.numel() * ws.element_size())
+
+
+def losa_block_mass(q: torch.Tensor, k: torch.Tensor, R: int, C: int, scale: Optional[float] = None,
+                    return_lse: bool = False, ws: Optional[torch.Tensor] = None,
+                    mass: Optional[torch.Tensor] = None):
+    """mass[B, H, nQb, nKb] (fp32) of one dense attention step; optionally the rows' log-sum-exp."""
+    _same_layout(q, k)
+    prob = make_problem(q, R, C, scale)
+    B, H, N, _ = q.shape
+    nQb, nKb = -(-N // R), -(-N // C)
+    if mass is None:
+        mass = torch.empty((B, H, nQb, nKb), dtype=torch.float32, device=q.device)
+    lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if return_lse else None
+    ws, ws_bytes = _workspace(LOSA_OP_BLOCK_MASS, prob, q.device, ws)
+    _check(_lib().losa_block_mass(ctypes.byref(prob), _ptr(q), _ptr(k), _ptr(mass), _ptr(lse),
+                                  _ptr(ws), ws_bytes, _stream()), "losa_block_mass")
+    return (mass, lse) if return_lse else mass
+
+
+def losa_select(mass: torch.Tensor, tau: float, kv_capacity: Optional[int] = None,
+                ws: Optional[torch.Tensor] = None,
+                out: Optional[Tuple[torch.Tensor, torch.Tensor]] = None):
+    """(offsets[rows + 1], kv_idx[kv_capacity]) int32; kv_idx is valid up to offsets[-1]."""
+    if mass.dim() != 4 or not mass.is_contiguous() or mass.dtype != torch.float32:
+        raise ValueError("mass must be a contiguous fp32 [B, H, nQb, nKb] tensor")
+    B, H, nQb, nKb = mass.shape
+    rows = B * H * nQb
+    if out is None:
+        cap = rows * nKb if kv_capacity is None else int(kv_capacity)
+        offsets = torch.empty(rows + 1, dtype=torch.int32, device=mass.device)
+        kv_idx = torch.empty(max(cap, 1), dtype=torch.int32, device=mass.device)
+    else:
+        offsets, kv_idx = out
+        cap = kv_idx.numel() if kv_capacity is None else int(kv_capacity)
+    ws_need = _select_workspace_bytes(B, H, nQb, nKb)
+    if ws is None:
+        ws = torch.empty(ws_need, dtype=torch.uint8, device=mass.device)
+    _check(_lib().losa_select(B, H, nQb, nKb, _ptr(mass), float(tau), _ptr(offsets), _ptr(kv_idx),
+                              cap, _ptr(ws), ws.numel(), _stream()), "losa_select")
+    return offsets, kv_idx
+
+
+def _select_workspace_bytes(B: int, H: int, nQb: int, nKb: int) -> int:
+    # losa_workspace_bytes(LOSA_OP_SELECT) reads B, H and ceil(N/R), ceil(N/C): describe the
+    # mass matrix as N = nQb * nKb tokens with R = nKb and C = nQb.
+    prob = Problem(B, H, nQb * nKb, 64, nKb, nQb, 0, 0, 0, 0.0)
+    return losa_workspace_bytes(LOSA_OP_SELECT, prob)
+
+
+def losa_sparse_attn(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, offsets: torch.Tensor,
+                     kv_idx: torch.Tensor, R: int, C: int, scale: Optional[float] = None,
+                     out_dtype: torch.dtype = torch.bfloat16, out: Optional[torch.Tensor] = None):
+    """Block-sparse attention over the frozen CSR pattern; rows >= N do not exist."""
+    _same_layout(q, k, v)
+    prob = make_problem(q, R, C, scale)
+    o = _alloc_out(q, out_dtype, out)
+    _check(_lib().losa_sparse_attn(ctypes.byref(prob), _ptr(q), _ptr(k), _ptr(v), _ptr(offsets),
+                                   _ptr(kv_idx), _ptr(o), _dtype_code(o.dtype), None, 0, _stream()),
+           "losa_sparse_attn")
+    return o
+
+
+def losa_attn(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, R: int = 128, C: int = 128,
+              scale: Optional[float] = None, out_dtype: torch.dtype = torch.bfloat16,
+              out: Optional[torch.Tensor] = None):
+    """Dense softmax attention with the library's own kernel."""
+    _same_layout(q, k, v)
+    prob = make_problem(q, R, C, scale)
+    o = _alloc_out(q, out_dtype, out)
+    _check(_lib().losa_attn(ctypes.byref(prob), _ptr(q), _ptr(k), _ptr(v), _ptr(o),
+                            _dtype_code(o.dtype), None, 0, _stream()), "losa_attn")
+    return o
+
+
+def losa_validate_csr(offsets: torch.Tensor, kv_idx: torch.Tensor, nKb: int) -> None:
+    _check(_lib().losa_validate_csr(offsets.numel() - 1, nKb, _ptr(offsets), _ptr(kv_idx), _stream()),
+           "losa_validate_csr")
+
+
+def losa_async_status() -> int:
+    """Synchronises the current stream and returns (and clears) the device-side status."""
+    return int(_lib().losa_async_status(_stream()))
+
+
+def losa_status_string(code: int) -> str:
+    return _lib().losa_status_string(code).decode()
+
+
+def check_async(where: str = "liblosa") -> None:
+    code = losa_async_status()
+    if code != 0:
+        raise LosaError(code, where)
+
+
+def _dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.bfloat16:
+        return LOSA_DTYPE_BF16
+    if dt == torch.float32:
+        return LOSA_DTYPE_F32
+    raise ValueError("output dtype must be bfloat16 or float32")
+
+
+def _alloc_out(q: torch.Tensor, dtype: torch.dtype, out: Optional[torch.Tensor]) -> torch.Tensor:
+    if out is not None:
+        if out.shape != q.shape or out.stride() != q.stride():
+            raise ValueError("o must share q's shape and strides")
+        return out
+    return torch.empty_strided(q.shape, q.stride(), dtype=dtype, device=q.device)
+
+
+def default_scale(D: int) -> float:
+    return 1.0 / math.sqrt(D)

@@ -1,0 +1,199 @@
+// C ABI of liblosa: argument validation, workspace sizing, status word, launch dispatch.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "losa_common.cuh"
+
+namespace losa {
+
+namespace {
+thread_local char g_cuda_error[256] = "";
+int* g_status_host = nullptr;
+int* g_status_dev = nullptr;
+}  // namespace
+
+const char* set_cuda_error(cudaError_t e, const char* what) {
+  snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", what, cudaGetErrorString(e));
+  return g_cuda_error;
+}
+
+// One pinned, mapped int per process; every CUDA device of a unified-addressing system can
+// reach it, so it is not per-device state.
+int* status_word_device() {
+  if (!g_status_dev) {
+    int* h = nullptr;
+    cudaError_t e = cudaHostAlloc(reinterpret_cast<void**>(&h), 64,
+                                  cudaHostAllocMapped | cudaHostAllocPortable);
+    if (e != cudaSuccess) {
+      set_cuda_error(e, "cudaHostAlloc(status word)");
+      return nullptr;
+    }
+    *h = 0;
+    int* d = nullptr;
+    e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&d), h, 0);
+    if (e != cudaSuccess) {
+      set_cuda_error(e, "cudaHostGetDevicePointer(status word)");
+      cudaFreeHost(h);
+      return nullptr;
+    }
+    g_status_host = h;
+    g_status_dev = d;
+  }
+  return g_status_dev;
+}
+
+int* status_word_host() { return g_status_host; }
+
+int make_geometry(const losa_problem_t* p, Geometry* g) {
+  if (!p) return LOSA_ERR_INVALID_ARG;
+  if (p->B <= 0 || p->H <= 0 || p->N <= 0) return LOSA_ERR_INVALID_ARG;
+  if (!(p->D == 64 || p->D == 128)) return LOSA_ERR_UNSUPPORTED;
+  if (!((p->R == 64 && p->C == 64) || (p->R == 128 && p->C == 128))) return LOSA_ERR_UNSUPPORTED;
+  if (p->sn < p->D || p->sh <= 0 || p->sb <= 0) return LOSA_ERR_INVALID_ARG;
+  if ((p->sn % 8) || (p->sh % 8) || (p->sb % 8)) return LOSA_ERR_INVALID_ARG;
+  if (!(p->scale >= 0.0f) || isinf(p->scale)) return LOSA_ERR_INVALID_ARG;
+  g->B = p->B;
+  g->H = p->H;
+  g->N = p->N;
+  g->D = p->D;
+  g->R = p->R;
+  g->C = p->C;
+  g->nQb = (p->N + p->R - 1) / p->R;
+  g->nKb = (p->N + p->C - 1) / p->C;
+  g->nQt = (p->N + 127) / 128;
+  g->nPairs = (g->nQt + 1) / 2;
+  g->sb = p->sb;
+  g->sh = p->sh;
+  g->sn = p->sn;
+  g->scale = (p->scale > 0.0f) ? p->scale : 1.0f / sqrtf((float)p->D);
+  const int64_t rows = (int64_t)g->B * g->H * g->nQb;
+  if (rows * g->nKb > INT32_MAX || (int64_t)g->B * g->H * g->nPairs > INT32_MAX)
+    return LOSA_ERR_UNSUPPORTED;
+  return LOSA_OK;
+}
+
+}  // namespace losa
+
+using namespace losa;
+
+extern "C" {
+
+size_t losa_workspace_bytes(int op, const losa_problem_t* p) {
+  if (!p) return 0;
+  if (op == LOSA_OP_SELECT) {
+    if (p->B <= 0 || p->H <= 0 || p->N <= 0 || p->R <= 0 || p->C <= 0) return 0;
+    const int64_t nQb = (p->N + p->R - 1) / p->R, nKb = (p->N + p->C - 1) / p->C;
+    return select_workspace_bytes((int64_t)p->B * p->H * nQb, (int)nKb);
+  }
+  Geometry g;
+  if (make_geometry(p, &g) != LOSA_OK) return 0;
+  switch (op) {
+    case LOSA_OP_BLOCK_MASS: return attn_workspace_bytes(kMass, g);
+    case LOSA_OP_SPARSE_ATTN: return attn_workspace_bytes(kSparse, g);
+    case LOSA_OP_ATTN: return attn_workspace_bytes(kDense, g);
+  }
+  return 0;
+}
+
+int losa_block_mass(const losa_problem_t* p, const void* q, const void* k, float* mass, float* lse,
+                    void* ws, size_t ws_bytes, void* cuda_stream) {
+  Geometry g;
+  int rc = make_geometry(p, &g);
+  if (rc != LOSA_OK) return rc;
+  if (!q || !k || !mass || !aligned16(q) || !aligned16(k) || !aligned16(mass))
+    return LOSA_ERR_INVALID_ARG;
+  const size_t need = attn_workspace_bytes(kMass, g);
+  if (need > 0 && (!ws || ws_bytes < need)) return LOSA_ERR_WORKSPACE;
+  if (!aligned16(ws)) return LOSA_ERR_INVALID_ARG;
+  return launch_attn(kMass, g, q, k, nullptr, nullptr, nullptr, nullptr, 0, mass, lse, ws,
+                     static_cast<cudaStream_t>(cuda_stream));
+}
+
+int losa_select(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const float* mass, double tau,
+                int32_t* offsets, int32_t* kv_idx, int64_t kv_capacity, void* ws, size_t ws_bytes,
+                void* cuda_stream) {
+  if (B <= 0 || H <= 0 || nQb <= 0 || nKb <= 0) return LOSA_ERR_INVALID_ARG;
+  if (!(tau > 0.0) || !(tau <= 1.0)) return LOSA_ERR_INVALID_ARG;  // also rejects NaN
+  if (!mass || !offsets || !kv_idx || kv_capacity < 0) return LOSA_ERR_INVALID_ARG;
+  const int64_t rows = (int64_t)B * H * nQb;
+  if (rows * nKb > INT32_MAX) return LOSA_ERR_UNSUPPORTED;
+  if (nKb > 8192) return LOSA_ERR_UNSUPPORTED;  // one row is sorted in shared memory
+  const size_t need = select_workspace_bytes(rows, nKb);
+  if (!ws || ws_bytes < need) return LOSA_ERR_WORKSPACE;
+  if (!aligned16(ws)) return LOSA_ERR_INVALID_ARG;
+  return launch_select((int)rows, nKb, mass, tau, offsets, kv_idx, kv_capacity, ws,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+static int check_attn_args(const losa_problem_t* p, Geometry* g, const void* q, const void* k,
+                           const void* v, const void* o, int o_dtype) {
+  int rc = make_geometry(p, g);
+  if (rc != LOSA_OK) return rc;
+  if (!q || !k || !v || !o) return LOSA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return LOSA_ERR_INVALID_ARG;
+  if (o_dtype != LOSA_DTYPE_BF16 && o_dtype != LOSA_DTYPE_F32) return LOSA_ERR_UNSUPPORTED;
+  return LOSA_OK;
+}
+
+int losa_sparse_attn(const losa_problem_t* p, const void* q, const void* k, const void* v,
+                     const int32_t* offsets, const int32_t* kv_idx, void* o, int o_dtype, void* ws,
+                     size_t ws_bytes, void* cuda_stream) {
+  (void)ws;
+  (void)ws_bytes;
+  Geometry g;
+  int rc = check_attn_args(p, &g, q, k, v, o, o_dtype);
+  if (rc != LOSA_OK) return rc;
+  if (!offsets || !kv_idx) return LOSA_ERR_INVALID_ARG;
+  return launch_attn(kSparse, g, q, k, v, offsets, kv_idx, o, o_dtype, nullptr, nullptr, nullptr,
+                     static_cast<cudaStream_t>(cuda_stream));
+}
+
+int losa_attn(const losa_problem_t* p, const void* q, const void* k, const void* v, void* o,
+              int o_dtype, void* ws, size_t ws_bytes, void* cuda_stream) {
+  (void)ws;
+  (void)ws_bytes;
+  Geometry g;
+  int rc = check_attn_args(p, &g, q, k, v, o, o_dtype);
+  if (rc != LOSA_OK) return rc;
+  return launch_attn(kDense, g, q, k, v, nullptr, nullptr, o, o_dtype, nullptr, nullptr, nullptr,
+                     static_cast<cudaStream_t>(cuda_stream));
+}
+
+int losa_validate_csr(int32_t rows, int32_t nKb, const int32_t* offsets, const int32_t* kv_idx,
+                      void* cuda_stream) {
+  if (rows <= 0 || nKb <= 0 || !offsets || !kv_idx) return LOSA_ERR_INVALID_ARG;
+  return launch_validate_csr(rows, nKb, offsets, kv_idx, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int losa_async_status(void* cuda_stream) {
+  cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) {
+    set_cuda_error(e, "cudaStreamSynchronize");
+    return LOSA_ERR_CUDA;
+  }
+  int* h = status_word_host();
+  if (!h) return LOSA_OK;  // nothing was ever launched
+  const int s = *reinterpret_cast<volatile int*>(h);
+  *reinterpret_cast<volatile int*>(h) = 0;
+  return s;
+}
+
+const char* losa_status_string(int status) {
+  switch (status) {
+    case LOSA_OK: return "LOSA_OK";
+    case LOSA_ERR_INVALID_ARG: return "LOSA_ERR_INVALID_ARG";
+    case LOSA_ERR_UNSUPPORTED: return "LOSA_ERR_UNSUPPORTED";
+    case LOSA_ERR_WORKSPACE: return "LOSA_ERR_WORKSPACE";
+    case LOSA_ERR_CAPACITY: return "LOSA_ERR_CAPACITY";
+    case LOSA_ERR_CUDA: return "LOSA_ERR_CUDA";
+    case LOSA_ERR_TIMEOUT: return "LOSA_ERR_TIMEOUT";
+    case LOSA_ERR_BAD_INDEX: return "LOSA_ERR_BAD_INDEX";
+    case LOSA_ERR_BAD_MASS: return "LOSA_ERR_BAD_MASS";
+  }
+  return "LOSA_ERR_UNKNOWN";
+}
+
+const char* losa_last_cuda_error(void) { return g_cuda_error; }
+
+}  // extern "C"

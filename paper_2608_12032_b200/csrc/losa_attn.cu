@@ -1,0 +1,745 @@
+// Attention kernels of liblosa for sm_100a: dense attention, block-sparse attention over a
+// frozen CSR pattern (Eq. 4) and the exact block-mass pass (Eq. 1), as ONE warp-specialised
+// persistent kernel template.
+//
+// CTA = 10 warps.  Warps 0-3 and 4-7 are two softmax warpgroups, each owning one 128-row
+// query tile (thread = query row = TMEM lane).  Warp 8 (one elected thread) is the TMA
+// producer: it streams the query tiles and the K / V tiles named by the block indices into
+// 128B-swizzled shared-memory rings.  Warp 9 (one elected thread) issues the tcgen05 MMAs:
+// S = Q K^T from shared memory into TMEM, O += P V with P read from TMEM (bf16, aliasing S)
+// and V from shared memory as the MN-major operand.
+//
+// A work item is a pair of consecutive query tiles of one (batch, head).  The key blocks the
+// pair visits are the ascending merge of the tiles' index lists (one list per query block;
+// two per tile when the block size is 64), so a K/V tile needed by both is loaded once, and
+// MMAs are issued only for the query tiles that list it.  Query-block rows that do not list
+// a tile of their 128-row group get P = 0 for it.
+//
+// The MMA thread runs one tile ahead on S: after O_t += P V(u) it issues S_t = Q_t K(u+1)^T
+// for the same tile t, then turns to the other tile, so each warpgroup's softmax overlaps
+// the other tile's MMAs.  Running maxima are updated lazily: O and the row sum are rescaled
+// only when the maximum grew by more than 2^8, which keeps the correction off the common
+// path without losing accuracy (the stale reference bounds p by 2^8).
+//
+// Every wait is bounded; a wait that expires raises the CTA's abort flag, records
+// LOSA_ERR_TIMEOUT, and all roles leave through the common teardown that frees TMEM.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <limits.h>
+#include <math.h>
+
+#include "losa_common.cuh"
+#include "losa_ptx.cuh"
+
+namespace losa {
+namespace {
+
+constexpr int kThreads = 320;
+constexpr int kTmemCols = 512;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.0f;
+
+template <int D, int BLK, int MODE>
+struct Cfg {
+  static constexpr int kC = BLK;                      // keys per K/V tile
+  static constexpr int kQBT = 128 / BLK;              // query blocks per 128-row tile
+  static constexpr int kNB = 2 * kQBT;                // query blocks per work item
+  static constexpr int kDH = D / 64;                  // 64-element slabs along D
+  static constexpr int kQSlab = 128 * 128;            // bytes of a [128][64] bf16 slab
+  static constexpr int kQBytes = kDH * kQSlab;        // one query tile
+  static constexpr int kKVSlab = kC * 128;            // bytes of a [C][64] bf16 slab
+  static constexpr int kKVBytes = kDH * kKVSlab;      // one K (or V) tile
+  static constexpr bool kHasV = (MODE != kMass);
+  static constexpr int kRingBudget = (kHasV ? 160 : 128) * 1024;  // K + V rings
+  static constexpr int kNV = kHasV ? ((kKVBytes >= 32768) ? 2 : 4) : 0;
+  static constexpr int kNK0 = (kRingBudget - kNV * kKVBytes) / kKVBytes;
+  static constexpr int kNK = kNK0 > 6 ? 6 : kNK0;
+  static constexpr uint32_t kIdescQK = ptx::idesc_bf16_f32(128, kC, false, false);
+  static constexpr uint32_t kIdescPV = ptx::idesc_bf16_f32(128, D, false, true);
+};
+
+struct Params {
+  int B, H, N, nQb, nKb, nQt, nPairs, nWork;
+  const int32_t* offsets;
+  const int32_t* kv_idx;
+  void* o;
+  int o_f32;
+  int64_t sb, sh, sn;
+  float* mass;
+  float* lse;
+  float2* table;  // mass mode: [grid][2][nKb][128] (sum of p, reference max) per row and tile
+  float scale_log2;
+  int* status;
+};
+
+template <int NK, int NV, bool MASS>
+struct Control {
+  uint64_t q_full[2], q_empty[2];
+  uint64_t k_full[NK], k_empty[NK];
+  uint64_t v_full[NV > 0 ? NV : 1], v_empty[NV > 0 ? NV : 1];
+  uint64_t s_full[2], p_ready[2], o_done[2], o_free[2];
+  uint64_t wg_bar[2];
+  uint64_t drain;
+  uint32_t tmem_base;
+  int abort_flag;
+  float2 rowstat[2][MASS ? 128 : 1];  // mass pass: final (max, 1/sum) of every row
+};
+
+// Ascending merge of the block-index lists of the (up to NB) query blocks of a work item.
+// Every role walks its own copy; the sequence is a pure function of the CSR, so they agree.
+template <int NB>
+struct TileIter {
+  const int32_t* idx;
+  int pos[NB], end[NB], cur[NB];
+  int nKb, dense_j;
+  uint32_t dense_mask;
+  bool dense;
+  int* status;
+
+  __device__ __forceinline__ void fetch(int n) {
+    cur[n] = INT_MAX;
+    while (pos[n] < end[n]) {
+      const int v = __ldg(idx + pos[n]);
+      if ((unsigned)v < (unsigned)nKb) {
+        cur[n] = v;
+        return;
+      }
+      report_error(status, LOSA_ERR_BAD_INDEX);  // skipped, never used as an address
+      ++pos[n];
+    }
+  }
+
+  __device__ __forceinline__ void init(const Params& p, bool is_dense, int bh, int first_block) {
+    idx = p.kv_idx;
+    nKb = p.nKb;
+    status = p.status;
+    dense = is_dense;
+    dense_j = 0;
+    dense_mask = 0;
+    const int32_t nnz = is_dense ? 0 : __ldg(p.offsets + (int64_t)p.B * p.H * p.nQb);
+#pragma unroll
+    for (int n = 0; n < NB; ++n) {
+      const int g = first_block + n;
+      pos[n] = end[n] = 0;
+      cur[n] = INT_MAX;
+      if (g < p.nQb) {
+        dense_mask |= 1u << n;
+        if (!is_dense) {
+          const int64_t row = (int64_t)bh * p.nQb + g;
+          const int32_t b = __ldg(p.offsets + row), e = __ldg(p.offsets + row + 1);
+          if (b < 0 || e < b || e > nnz || e - b > p.nKb) {
+            report_error(status, LOSA_ERR_BAD_INDEX);
+          } else {
+            pos[n] = b;
+            end[n] = e;
+            fetch(n);
+          }
+        }
+      }
+    }
+  }
+
+  __device__ __forceinline__ bool next(int& j, uint32_t& memb) {
+    if (dense) {
+      if (dense_j >= nKb || dense_mask == 0) return false;
+      j = dense_j++;
+      memb = dense_mask;
+      return true;
+    }
+    int m = INT_MAX;
+#pragma unroll
+    for (int n = 0; n < NB; ++n) m = min(m, cur[n]);
+    if (m == INT_MAX) return false;
+    memb = 0;
+#pragma unroll
+    for (int n = 0; n < NB; ++n) {
+      if (cur[n] == m) {
+        memb |= 1u << n;
+        ++pos[n];
+        fetch(n);
+      }
+    }
+    j = m;
+    return true;
+  }
+};
+
+#define LOSA_WAIT(bar, parity)                                   \
+  do {                                                           \
+    if (!ptx::mbar_wait((bar), (parity), &ctl->abort_flag)) {    \
+      ctl->abort_flag = 1;                                       \
+      report_error(p.status, LOSA_ERR_TIMEOUT);                  \
+      goto teardown;                                             \
+    }                                                            \
+  } while (0)
+
+template <int D, int BLK, int MODE>
+__global__ void __launch_bounds__(kThreads, 1)
+losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                 const __grid_constant__ CUtensorMap map_v, const Params p) {
+  using C = Cfg<D, BLK, MODE>;
+  using Ctl = Control<C::kNK, C::kNV, MODE == kMass>;
+  constexpr int kC = C::kC, kQBT = C::kQBT, kNB = C::kNB;
+  constexpr uint32_t kQMask = (1u << kQBT) - 1u;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                             ~static_cast<uintptr_t>(1023));
+  uint8_t* sQ = smem;
+  uint8_t* sK = sQ + 2 * C::kQBytes;
+  uint8_t* sV = sK + C::kNK * C::kKVBytes;
+  Ctl* ctl = reinterpret_cast<Ctl*>(sV + C::kNV * C::kKVBytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(&ctl->q_full[i], 1);
+      ptx::mbar_init(&ctl->q_empty[i], 1);
+      ptx::mbar_init(&ctl->s_full[i], 1);
+      ptx::mbar_init(&ctl->p_ready[i], 128);
+      ptx::mbar_init(&ctl->o_done[i], 1);
+      ptx::mbar_init(&ctl->o_free[i], 128);
+      ptx::mbar_init(&ctl->wg_bar[i], 128);
+    }
+    for (int i = 0; i < C::kNK; ++i) {
+      ptx::mbar_init(&ctl->k_full[i], 1);
+      ptx::mbar_init(&ctl->k_empty[i], 1);
+    }
+    for (int i = 0; i < C::kNV; ++i) {
+      ptx::mbar_init(&ctl->v_full[i], 1);
+      ptx::mbar_init(&ctl->v_empty[i], 1);
+    }
+    ptx::mbar_init(&ctl->drain, 1);
+    ctl->abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  if (warp == 9) {
+    ptx::tmem_alloc(&ctl->tmem_base, kTmemCols);
+    ptx::tmem_relinquish_alloc_permit();
+  }
+  if (warp == 8 && lane == 0) {
+    ptx::prefetch_tensormap(&map_q);
+    ptx::prefetch_tensormap(&map_k);
+    if (C::kHasV) ptx::prefetch_tensormap(&map_v);
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = ctl->tmem_base;
+
+  if (warp == 8) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t nq[2] = {0, 0}, nk = 0, nv = 0;
+      for (int w = blockIdx.x; w < p.nWork; w += gridDim.x) {
+        const int bh = w / p.nPairs, pr = w % p.nPairs;
+        const int b = bh / p.H, h = bh % p.H;
+#pragma unroll
+        for (int qt = 0; qt < 2; ++qt) {
+          const int T = 2 * pr + qt;
+          if (T < p.nQt) {
+            LOSA_WAIT(&ctl->q_empty[qt], (nq[qt] & 1) ^ 1);
+            ptx::mbar_arrive_expect_tx(&ctl->q_full[qt], C::kQBytes);
+#pragma unroll
+            for (int s = 0; s < C::kDH; ++s)
+              ptx::tma_load_4d(sQ + qt * C::kQBytes + s * C::kQSlab, &map_q, &ctl->q_full[qt],
+                               s * 64, T * 128, h, b);
+            ++nq[qt];
+          }
+        }
+        TileIter<kNB> it;
+        it.init(p, MODE != kSparse, bh, 2 * pr * kQBT);
+        int j;
+        uint32_t memb;
+        while (it.next(j, memb)) {
+          const uint32_t ks = nk % C::kNK;
+          LOSA_WAIT(&ctl->k_empty[ks], ((nk / C::kNK) & 1) ^ 1);
+          ptx::mbar_arrive_expect_tx(&ctl->k_full[ks], C::kKVBytes);
+#pragma unroll
+          for (int s = 0; s < C::kDH; ++s)
+            ptx::tma_load_4d(sK + ks * C::kKVBytes + s * C::kKVSlab, &map_k, &ctl->k_full[ks],
+                             s * 64, j * kC, h, b);
+          ++nk;
+          if (C::kHasV) {
+            const uint32_t vs = nv % (C::kNV > 0 ? C::kNV : 1);
+            LOSA_WAIT(&ctl->v_empty[vs], ((nv / (C::kNV > 0 ? C::kNV : 1)) & 1) ^ 1);
+            ptx::mbar_arrive_expect_tx(&ctl->v_full[vs], C::kKVBytes);
+#pragma unroll
+            for (int s = 0; s < C::kDH; ++s)
+              ptx::tma_load_4d(sV + vs * C::kKVBytes + s * C::kKVSlab, &map_v, &ctl->v_full[vs],
+                               s * 64, j * kC, h, b);
+            ++nv;
+          }
+        }
+      }
+    }
+  } else if (warp == 9) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t q_base = ptx::smem_u32(sQ), k_base = ptx::smem_u32(sK),
+                     v_base = ptx::smem_u32(sV);
+      uint32_t nq[2] = {0, 0}, nk = 0, nv = 0, np[2] = {0, 0}, nof[2] = {0, 0};
+
+      auto issue_qk = [&](int qt, uint32_t ks) {
+        const uint32_t a0 = q_base + qt * C::kQBytes, b0 = k_base + ks * C::kKVBytes;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk & 3) * 32;
+          const uint64_t ad = ptx::smem_desc_sw128(a0 + (kk >> 2) * C::kQSlab + off, 16, 1024);
+          const uint64_t bd = ptx::smem_desc_sw128(b0 + (kk >> 2) * C::kKVSlab + off, 16, 1024);
+          ptx::mma_ss(tmem_base + qt * 128, ad, bd, C::kIdescQK, kk > 0 ? 1u : 0u);
+        }
+      };
+      auto issue_pv = [&](int qt, uint32_t vs, bool accumulate) {
+        const uint32_t b0 = v_base + vs * C::kKVBytes;
+#pragma unroll
+        for (int kk = 0; kk < kC / 16; ++kk) {
+          const uint64_t bd = ptx::smem_desc_sw128(b0 + kk * 2048, C::kKVSlab, 1024);
+          ptx::mma_ts(tmem_base + 256 + qt * 128, tmem_base + qt * 128 + kk * 8, bd, C::kIdescPV,
+                      (accumulate || kk > 0) ? 1u : 0u);
+        }
+      };
+
+      for (int w = blockIdx.x; w < p.nWork; w += gridDim.x) {
+        const int bh = w / p.nPairs, pr = w % p.nPairs;
+        TileIter<kNB> it;
+        it.init(p, MODE != kSparse, bh, 2 * pr * kQBT);
+        bool q_ready[2] = {false, false};
+        uint32_t pv_item[2] = {0, 0};
+        int jc;
+        uint32_t mc;
+        bool have = it.next(jc, mc);
+        if (have) {
+          const uint32_t ks = nk % C::kNK;
+          LOSA_WAIT(&ctl->k_full[ks], (nk / C::kNK) & 1);
+#pragma unroll
+          for (int qt = 0; qt < 2; ++qt) {
+            if ((mc >> (qt * kQBT)) & kQMask) {
+              LOSA_WAIT(&ctl->q_full[qt], nq[qt] & 1);
+              ++nq[qt];
+              q_ready[qt] = true;
+              ptx::tc_fence_after_sync();
+              issue_qk(qt, ks);
+              ptx::mma_commit(&ctl->s_full[qt]);
+            }
+          }
+          ptx::mma_commit(&ctl->k_empty[ks]);
+          ++nk;
+        }
+        while (have) {
+          int jn;
+          uint32_t mn;
+          const bool have_n = it.next(jn, mn);
+          const uint32_t ksn = nk % C::kNK;
+          const uint32_t vs = nv % (C::kNV > 0 ? C::kNV : 1);
+          if (have_n) LOSA_WAIT(&ctl->k_full[ksn], (nk / C::kNK) & 1);
+          if (C::kHasV) LOSA_WAIT(&ctl->v_full[vs], (nv / (C::kNV > 0 ? C::kNV : 1)) & 1);
+#pragma unroll
+          for (int qt = 0; qt < 2; ++qt) {
+            if ((mc >> (qt * kQBT)) & kQMask) {
+              LOSA_WAIT(&ctl->p_ready[qt], np[qt] & 1);
+              ++np[qt];
+              if (C::kHasV) {
+                if (pv_item[qt] == 0 && nof[qt] > 0)
+                  LOSA_WAIT(&ctl->o_free[qt], (nof[qt] - 1) & 1);
+                ptx::tc_fence_after_sync();
+                issue_pv(qt, vs, pv_item[qt] > 0);
+                ptx::mma_commit(&ctl->o_done[qt]);
+                ++pv_item[qt];
+              }
+            }
+            if (have_n && ((mn >> (qt * kQBT)) & kQMask)) {
+              if (!q_ready[qt]) {
+                LOSA_WAIT(&ctl->q_full[qt], nq[qt] & 1);
+                ++nq[qt];
+                q_ready[qt] = true;
+              }
+              ptx::tc_fence_after_sync();
+              issue_qk(qt, ksn);
+              ptx::mma_commit(&ctl->s_full[qt]);
+            }
+          }
+          if (C::kHasV) {
+            ptx::mma_commit(&ctl->v_empty[vs]);
+            ++nv;
+          }
+          if (have_n) {
+            ptx::mma_commit(&ctl->k_empty[ksn]);
+            ++nk;
+          }
+          have = have_n;
+          mc = mn;
+          jc = jn;
+        }
+#pragma unroll
+        for (int qt = 0; qt < 2; ++qt) {
+          if (q_ready[qt]) ptx::mma_commit(&ctl->q_empty[qt]);
+          if (pv_item[qt] > 0) ++nof[qt];
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax warpgroups
+    const int qt = warp >> 2, wl = warp & 3;
+    const int row = wl * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(wl * 32) << 16;
+    const uint32_t tS = tmem_base + lane_base + qt * 128;
+    const uint32_t tO = tmem_base + lane_base + 256 + qt * 128;
+    const int sub = (BLK == 64) ? (wl >> 1) : 0;
+    const int my_bit = qt * kQBT + sub;
+    const int tail = p.N - (p.nKb - 1) * kC;  // valid keys of the last K/V tile
+    uint32_t ns = 0, npv = 0, nwg = 0;
+
+    for (int w = blockIdx.x; w < p.nWork; w += gridDim.x) {
+      const int bh = w / p.nPairs, pr = w % p.nPairs;
+      const int b = bh / p.H, h = bh % p.H;
+      const int T = 2 * pr + qt;
+      const int grow = T * 128 + row;
+      TileIter<kNB> it;
+      it.init(p, MODE != kSparse, bh, 2 * pr * kQBT);
+      float m_ref = -INFINITY, l = 0.f;
+      uint32_t pv_item = 0;
+      float2* tab = nullptr;
+      if (MODE == kMass)
+        tab = p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * 128 + row;
+      int j;
+      uint32_t memb;
+      while (it.next(j, memb)) {
+        if (((memb >> (qt * kQBT)) & kQMask) == 0) continue;
+        LOSA_WAIT(&ctl->s_full[qt], ns & 1);
+        ++ns;
+        ptx::tc_fence_after_sync();
+        const bool mine = (memb >> my_bit) & 1u;
+        if (mine) {
+          uint32_t sr[kC];
+#pragma unroll
+          for (int c0 = 0; c0 < kC; c0 += 32) ptx::tmem_ld32(tS + c0, &sr[c0]);
+          ptx::tmem_wait_ld();
+          float s[kC];
+#pragma unroll
+          for (int c = 0; c < kC; ++c) s[c] = __uint_as_float(sr[c]);
+          if (j == p.nKb - 1 && tail < kC) {
+#pragma unroll
+            for (int c = 0; c < kC; ++c)
+              if (c >= tail) s[c] = -INFINITY;
+          }
+          float mx0 = s[0], mx1 = s[1], mx2 = s[2], mx3 = s[3];
+#pragma unroll
+          for (int c = 4; c < kC; c += 4) {
+            mx0 = fmaxf(mx0, s[c]);
+            mx1 = fmaxf(mx1, s[c + 1]);
+            mx2 = fmaxf(mx2, s[c + 2]);
+            mx3 = fmaxf(mx3, s[c + 3]);
+          }
+          const float m_new = fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
+          const bool need = m_new > m_ref + kRescaleThreshold;
+          if (__any_sync(0xffffffffu, need)) {
+            const float alpha = need ? ptx::ex2_approx(m_ref - m_new) : 1.f;
+            if (need) m_ref = m_new;
+            l *= alpha;
+            if (C::kHasV && pv_item > 0) {
+              LOSA_WAIT(&ctl->o_done[qt], (npv - 1) & 1);
+              ptx::tc_fence_after_sync();
+#pragma unroll
+              for (int c0 = 0; c0 < D; c0 += 32) {
+                uint32_t r[32];
+                ptx::tmem_ld32(tO + c0, r);
+                ptx::tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
+                ptx::tmem_st32(tO + c0, r);
+              }
+            }
+          }
+          float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+          const float neg_m = -m_ref;
+#pragma unroll
+          for (int c = 0; c < kC; c += 4) {
+            s[c] = ptx::ex2_approx(fmaf(s[c], p.scale_log2, neg_m));
+            s[c + 1] = ptx::ex2_approx(fmaf(s[c + 1], p.scale_log2, neg_m));
+            s[c + 2] = ptx::ex2_approx(fmaf(s[c + 2], p.scale_log2, neg_m));
+            s[c + 3] = ptx::ex2_approx(fmaf(s[c + 3], p.scale_log2, neg_m));
+            l0 += s[c];
+            l1 += s[c + 1];
+            l2 += s[c + 2];
+            l3 += s[c + 3];
+          }
+          const float tsum = (l0 + l1) + (l2 + l3);
+          l += tsum;
+          if (C::kHasV) {
+#pragma unroll
+            for (int c0 = 0; c0 < kC / 2; c0 += 32) {
+              uint32_t pk[32];
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                pk[c] = ptx::pack_bf16x2(s[2 * (c0 + c)], s[2 * (c0 + c) + 1]);
+              ptx::tmem_st32(tS + c0, pk);
+            }
+          } else {
+            tab[(int64_t)j * 128] = make_float2(tsum, m_ref);
+          }
+        } else if (C::kHasV) {
+          uint32_t z[32];
+#pragma unroll
+          for (int c = 0; c < 32; ++c) z[c] = 0u;
+#pragma unroll
+          for (int c0 = 0; c0 < kC / 2; c0 += 32) ptx::tmem_st32(tS + c0, z);
+        }
+        if (C::kHasV) {
+          ptx::tmem_wait_st();
+          ++pv_item;
+          ++npv;
+        }
+        ptx::tc_fence_before_sync();
+        ptx::mbar_arrive(&ctl->p_ready[qt]);
+      }
+
+      if (MODE != kMass) {
+        // ---- epilogue: O / l -> global
+        if (T < p.nQt) {
+          const bool valid = grow < p.N;
+          const float inv = (l > 0.f) ? 1.f / l : 0.f;
+          const int64_t off = (int64_t)b * p.sb + (int64_t)h * p.sh + (int64_t)grow * p.sn;
+          if (pv_item > 0) {
+            LOSA_WAIT(&ctl->o_done[qt], (npv - 1) & 1);
+            ptx::tc_fence_after_sync();
+          }
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 32) {
+            uint32_t r[32];
+            if (pv_item > 0) {
+              ptx::tmem_ld32(tO + c0, r);
+              ptx::tmem_wait_ld();
+            } else {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) r[c] = 0u;
+            }
+            if (valid) {
+              if (p.o_f32) {
+                float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + off + c0);
+#pragma unroll
+                for (int c = 0; c < 32; c += 4)
+                  dst[c >> 2] = make_float4(__uint_as_float(r[c]) * inv, __uint_as_float(r[c + 1]) * inv,
+                                            __uint_as_float(r[c + 2]) * inv,
+                                            __uint_as_float(r[c + 3]) * inv);
+              } else {
+                uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.o) + off + c0);
+#pragma unroll
+                for (int c = 0; c < 32; c += 8) {
+                  uint4 v;
+                  v.x = ptx::pack_bf16x2(__uint_as_float(r[c]) * inv, __uint_as_float(r[c + 1]) * inv);
+                  v.y = ptx::pack_bf16x2(__uint_as_float(r[c + 2]) * inv, __uint_as_float(r[c + 3]) * inv);
+                  v.z = ptx::pack_bf16x2(__uint_as_float(r[c + 4]) * inv, __uint_as_float(r[c + 5]) * inv);
+                  v.w = ptx::pack_bf16x2(__uint_as_float(r[c + 6]) * inv, __uint_as_float(r[c + 7]) * inv);
+                  dst[c >> 3] = v;
+                }
+              }
+            }
+          }
+          if (pv_item > 0) {
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(&ctl->o_free[qt]);
+          }
+        }
+      } else {
+        // ---- epilogue of the mass pass: normalise the per-tile sums by the final row
+        // statistics and average them over the rows of each query block
+        if (T < p.nQt) {
+          const bool valid = grow < p.N;
+          ctl->rowstat[qt][row] = make_float2(m_ref, (valid && l > 0.f) ? 1.f / l : 0.f);
+          if (p.lse != nullptr && valid)
+            p.lse[(int64_t)bh * p.N + grow] = (m_ref + log2f(l)) * kLn2;
+        }
+        ptx::mbar_arrive(&ctl->wg_bar[qt]);  // warpgroup sync with a bounded wait
+        LOSA_WAIT(&ctl->wg_bar[qt], nwg & 1);
+        ++nwg;
+        if (T < p.nQt) {
+          const float2* tb = p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * 128;
+          for (int u = wl; u < p.nKb; u += 4) {
+            float acc[kQBT];
+#pragma unroll
+            for (int q = 0; q < kQBT; ++q) acc[q] = 0.f;
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr) {
+              const int r = rr * 32 + lane;
+              const float2 tv = tb[(int64_t)u * 128 + r];
+              const float2 st = ctl->rowstat[qt][r];
+              const float wgt = (st.y > 0.f) ? tv.x * ptx::ex2_approx(tv.y - st.x) * st.y : 0.f;
+              acc[(rr * 32) / BLK] += wgt;
+            }
+#pragma unroll
+            for (int q = 0; q < kQBT; ++q) {
+              float a = acc[q];
+#pragma unroll
+              for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
+              const int g = T * kQBT + q;
+              if (lane == 0 && g < p.nQb) {
+                const int nvalid = min(BLK, p.N - g * BLK);
+                p.mass[((int64_t)bh * p.nQb + g) * p.nKb + u] = a / (float)nvalid;
+              }
+            }
+          }
+        }
+        ptx::mbar_arrive(&ctl->wg_bar[qt]);
+        LOSA_WAIT(&ctl->wg_bar[qt], nwg & 1);
+        ++nwg;
+      }
+    }
+  }
+
+teardown:
+  if (ctl->abort_flag) {
+    // Abort path: give MMAs and bulk copies still in flight a bounded time to land before
+    // shared memory and TMEM are released.
+    if (warp == 9 && lane == 0) {
+      ptx::mma_commit(&ctl->drain);
+      for (uint32_t it = 0; it < (1u << 16); ++it) {
+        if (ptx::mbar_try_wait(&ctl->drain, 0)) break;
+        __nanosleep(128);
+      }
+    }
+    if (warp == 8 && lane == 0) {
+      for (uint32_t it = 0; it < (1u << 10); ++it) __nanosleep(1024);
+    }
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 9) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+#undef LOSA_WAIT
+
+// ---------------------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) ==
+            cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  return fn;
+}
+
+// bf16 [B,H,N,D] tensor, box = [box_rows][64] with 128-byte swizzle; rows >= N read as zero.
+int make_map(CUtensorMap* m, const void* base, const Geometry& g, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) {
+    set_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled entry point");
+    return LOSA_ERR_CUDA;
+  }
+  const cuuint64_t dims[4] = {(cuuint64_t)g.D, (cuuint64_t)g.N, (cuuint64_t)g.H, (cuuint64_t)g.B};
+  const cuuint64_t strides[3] = {(cuuint64_t)g.sn * 2, (cuuint64_t)g.sh * 2, (cuuint64_t)g.sb * 2};
+  const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
+                        strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    return LOSA_ERR_CUDA;
+  }
+  return LOSA_OK;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
+  }
+  return n;
+}
+
+template <int D, int BLK, int MODE>
+int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Params prm,
+             cudaStream_t st) {
+  using C = Cfg<D, BLK, MODE>;
+  using Ctl = Control<C::kNK, C::kNV, MODE == kMass>;
+  CUtensorMap mq, mk, mv;
+  int rc;
+  if ((rc = make_map(&mq, q, g, 128)) != LOSA_OK) return rc;
+  if ((rc = make_map(&mk, k, g, C::kC)) != LOSA_OK) return rc;
+  if ((rc = make_map(&mv, C::kHasV ? v : k, g, C::kC)) != LOSA_OK) return rc;
+  const size_t smem =
+      1024 + 2 * C::kQBytes + (size_t)(C::kNK + C::kNV) * C::kKVBytes + sizeof(Ctl);
+  auto kern = losa_attn_kernel<D, BLK, MODE>;
+  static bool configured = false;
+  if (!configured) {
+    LOSA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    configured = true;
+  }
+  int sms = sm_count();
+  if (sms <= 0) return LOSA_ERR_CUDA;
+  const int grid = min(min(sms, kMaxPersistentCtas), prm.nWork);
+  kern<<<grid, kThreads, smem, st>>>(mq, mk, mv, prm);
+  LOSA_CUDA_TRY(cudaGetLastError());
+  return LOSA_OK;
+}
+
+template <int MODE>
+int dispatch(const Geometry& g, const void* q, const void* k, const void* v, const Params& prm,
+             cudaStream_t st) {
+  if (g.D == 128 && g.R == 128) return launch_t<128, 128, MODE>(g, q, k, v, prm, st);
+  if (g.D == 64 && g.R == 64) return launch_t<64, 64, MODE>(g, q, k, v, prm, st);
+  if (g.D == 128 && g.R == 64) return launch_t<128, 64, MODE>(g, q, k, v, prm, st);
+  if (g.D == 64 && g.R == 128) return launch_t<64, 128, MODE>(g, q, k, v, prm, st);
+  return LOSA_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+size_t attn_workspace_bytes(AttnMode mode, const Geometry& g) {
+  if (mode != kMass) return 0;
+  return (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2);
+}
+
+int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, const void* v,
+                const int32_t* offsets, const int32_t* kv_idx, void* o, int o_dtype, float* mass,
+                float* lse, void* ws, cudaStream_t st) {
+  Params prm;
+  prm.B = g.B;
+  prm.H = g.H;
+  prm.N = g.N;
+  prm.nQb = g.nQb;
+  prm.nKb = g.nKb;
+  prm.nQt = g.nQt;
+  prm.nPairs = g.nPairs;
+  prm.nWork = g.B * g.H * g.nPairs;
+  prm.offsets = offsets;
+  prm.kv_idx = kv_idx;
+  prm.o = o;
+  prm.o_f32 = (o_dtype == LOSA_DTYPE_F32) ? 1 : 0;
+  prm.sb = g.sb;
+  prm.sh = g.sh;
+  prm.sn = g.sn;
+  prm.mass = mass;
+  prm.lse = lse;
+  prm.table = static_cast<float2*>(ws);
+  prm.scale_log2 = g.scale * kLog2e;
+  prm.status = status_word_device();
+  if (!prm.status) return LOSA_ERR_CUDA;
+  switch (mode) {
+    case kDense: return dispatch<kDense>(g, q, k, v, prm, st);
+    case kSparse: return dispatch<kSparse>(g, q, k, v, prm, st);
+    case kMass: return dispatch<kMass>(g, q, k, v, prm, st);
+  }
+  return LOSA_ERR_INVALID_ARG;
+}
+
+}  // namespace losa

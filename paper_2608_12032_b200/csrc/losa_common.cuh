@@ -1,0 +1,62 @@
+// Shared host/device helpers of liblosa: status word, problem geometry, error macros.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "losa.h"
+
+namespace losa {
+
+// Upper bound on the number of persistent CTAs any kernel here launches; workspace is
+// sized for it so that losa_workspace_bytes() needs no GPU.
+constexpr int kMaxPersistentCtas = 160;
+
+// Device-visible status word (pinned, mapped host memory).  Kernels record the first
+// error with a system-scope compare-and-swap; the host reads it after a stream sync.
+int* status_word_device();  // device pointer, valid on the current device
+int* status_word_host();
+const char* set_cuda_error(cudaError_t e, const char* what);
+
+__device__ __forceinline__ void report_error(int* status, int code) {
+  atomicCAS_system(status, 0, code);
+}
+
+struct Geometry {
+  int B, H, N, D, R, C;
+  int nQb, nKb;
+  int nQt;     // 128-row query tiles per head
+  int nPairs;  // pairs of query tiles per head (one CTA work item)
+  int64_t sb, sh, sn;
+  float scale;
+};
+
+int make_geometry(const losa_problem_t* p, Geometry* g);  // LOSA_OK or an error code
+
+#define LOSA_CUDA_TRY(expr)                                        \
+  do {                                                             \
+    cudaError_t e__ = (expr);                                      \
+    if (e__ != cudaSuccess) {                                      \
+      ::losa::set_cuda_error(e__, #expr);                          \
+      return LOSA_ERR_CUDA;                                        \
+    }                                                              \
+  } while (0)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ---- entry points of the kernel translation units (host launchers) -------------------
+
+size_t select_workspace_bytes(int64_t rows, int nKb);
+int launch_select(int rows, int nKb, const float* mass, double tau, int32_t* offsets,
+                  int32_t* kv_idx, int64_t kv_capacity, void* ws, cudaStream_t st);
+int launch_validate_csr(int rows, int nKb, const int32_t* offsets, const int32_t* kv_idx,
+                        cudaStream_t st);
+
+enum AttnMode { kDense = 0, kSparse = 1, kMass = 2 };
+
+size_t attn_workspace_bytes(AttnMode mode, const Geometry& g);
+int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, const void* v,
+                const int32_t* offsets, const int32_t* kv_idx, void* o, int o_dtype, float* mass,
+                float* lse, void* ws, cudaStream_t st);
+
+}  // namespace losa

@@ -1,0 +1,245 @@
+// losa_select: retained-mass selection (Eq. 3) and CSR validation.
+//
+// Three small launches over a [rows, nKb] fp32 mass matrix:
+//   1. select_rows_kernel   one CTA per row: sort (mass descending, index ascending) as
+//                           64-bit integer keys in shared memory, fp64 prefix sum along the
+//                           sorted order, shortest prefix reaching tau; the kept set is
+//                           written as a bitmap over block indices plus its size.
+//   2. scan_counts_kernel   exclusive prefix of the per-row sizes -> offsets.
+//   3. expand_rows_kernel   one warp per row: bitmap -> ascending block indices.
+// Each mass element is read once and each kept index written once; the bitmap adds 1/16
+// of the mass bytes.  The result is deterministic (no floating-point atomics).
+#include <limits.h>
+
+#include "losa_common.cuh"
+
+namespace losa {
+namespace {
+
+constexpr int kSelThreads = 256;
+constexpr unsigned long long kPadKey = ~0ull;
+
+__device__ __forceinline__ double key_mass(unsigned long long key) {
+  return (double)__uint_as_float(~(uint32_t)(key >> 32));
+}
+
+__global__ void __launch_bounds__(kSelThreads)
+select_rows_kernel(const float* __restrict__ mass, int nKb, int n2, double tau,
+                   int32_t* __restrict__ counts, uint32_t* __restrict__ bitmaps, int* status) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);
+  uint32_t* bitmap = reinterpret_cast<uint32_t*>(keys + n2);
+  __shared__ double warp_total[kSelThreads / 32];
+  __shared__ int first_pos;
+
+  const int tid = threadIdx.x;
+  const int64_t row = blockIdx.x;
+  const int words = (nKb + 31) >> 5;
+  const float* mrow = mass + row * nKb;
+
+  bool bad = false;
+  for (int i = tid; i < n2; i += kSelThreads) {
+    unsigned long long key = kPadKey;
+    if (i < nKb) {
+      float m = mrow[i];
+      if (!(m >= 0.0f)) {  // negative or NaN
+        bad = true;
+        m = 0.0f;
+      }
+      // mass >= 0, so its IEEE bits order like the value; -0 becomes +0
+      const uint32_t bits = (m == 0.0f) ? 0u : __float_as_uint(m);
+      key = ((unsigned long long)(~bits) << 32) | (uint32_t)i;
+    }
+    keys[i] = key;
+  }
+  for (int w = tid; w < words; w += kSelThreads) bitmap[w] = 0u;
+  if (tid == 0) first_pos = INT_MAX;
+  if (bad) report_error(status, LOSA_ERR_BAD_MASS);
+  __syncthreads();
+
+  // bitonic sort, ascending keys = descending mass, ties by ascending block index
+  for (int k = 2; k <= n2; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int i = tid; i < n2; i += kSelThreads) {
+        const int ixj = i ^ j;
+        if (ixj > i) {
+          const unsigned long long a = keys[i], b = keys[ixj];
+          const bool up = ((i & k) == 0);
+          if ((a > b) == up) {
+            keys[i] = b;
+            keys[ixj] = a;
+          }
+        }
+      }
+      __syncthreads();
+    }
+  }
+
+  // fp64 prefix sum along the sorted order: per-thread chunk, then a block scan of chunk sums
+  const int chunk = (n2 + kSelThreads - 1) / kSelThreads;
+  const int lo = min(tid * chunk, n2), hi = min(lo + chunk, n2);
+  double local = 0.0;
+  for (int i = lo; i < hi; ++i) local += key_mass(keys[i]);
+  double incl = local;
+  const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const double up = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += up;
+  }
+  if (lane == 31) warp_total[warp] = incl;
+  __syncthreads();
+  double base = 0.0;
+  for (int w = 0; w < warp; ++w) base += warp_total[w];
+  double acc = base + (incl - local);
+  for (int i = lo; i < hi; ++i) {
+    acc += key_mass(keys[i]);
+    if (acc >= tau) {
+      atomicMin(&first_pos, i + 1);
+      break;
+    }
+  }
+  __syncthreads();
+  int s = first_pos;
+  if (tau >= 1.0 || s > nKb) s = nKb;
+
+  for (int i = lo; i < hi; ++i) {
+    if (i < s) {
+      const uint32_t idx = (uint32_t)keys[i];
+      atomicOr(&bitmap[idx >> 5], 1u << (idx & 31));
+    }
+  }
+  __syncthreads();
+  for (int w = tid; w < words; w += kSelThreads) bitmaps[row * words + w] = bitmap[w];
+  if (tid == 0) counts[row] = s;
+}
+
+__global__ void __launch_bounds__(1024)
+scan_counts_kernel(const int32_t* __restrict__ counts, int rows, int32_t* __restrict__ offsets,
+                   int64_t kv_capacity, int* status) {
+  __shared__ int warp_total[32];
+  __shared__ int carry_s;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) carry_s = 0;
+  __syncthreads();
+  for (int base = 0; base < rows; base += 1024) {
+    const int i = base + tid;
+    const int c = (i < rows) ? counts[i] : 0;
+    int incl = c;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += up;
+    }
+    if (lane == 31) warp_total[warp] = incl;
+    __syncthreads();
+    int wbase = 0;
+    for (int w = 0; w < warp; ++w) wbase += warp_total[w];
+    const int carry = carry_s;
+    if (i < rows) offsets[i] = carry + wbase + incl - c;
+    __syncthreads();
+    if (tid == 1023) carry_s = carry + wbase + incl;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    offsets[rows] = carry_s;
+    if ((int64_t)carry_s > kv_capacity) report_error(status, LOSA_ERR_CAPACITY);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+expand_rows_kernel(const uint32_t* __restrict__ bitmaps, const int32_t* __restrict__ offsets,
+                   int rows, int nKb, int32_t* __restrict__ kv_idx, int64_t kv_capacity) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const int words = (nKb + 31) >> 5;
+  int64_t pos0 = offsets[row];
+  for (int w0 = 0; w0 < words; w0 += 32) {
+    const int w = w0 + lane;
+    uint32_t word = (w < words) ? bitmaps[row * words + w] : 0u;
+    const int cnt = __popc(word);
+    int incl = cnt;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += up;
+    }
+    int64_t pos = pos0 + incl - cnt;
+    while (word) {
+      const int b = __ffs(word) - 1;
+      word &= word - 1;
+      if (pos < kv_capacity) kv_idx[pos] = w * 32 + b;
+      ++pos;
+    }
+    pos0 += __shfl_sync(0xffffffffu, incl, 31);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+validate_csr_kernel(int rows, int nKb, const int32_t* __restrict__ offsets,
+                    const int32_t* __restrict__ kv_idx, int* status) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const int32_t b = offsets[row], e = offsets[row + 1];
+  const int32_t nnz = offsets[rows];  // every read below stays inside [0, nnz)
+  bool bad = (row == 0 && b != 0) || e <= b || (e - b) > nKb || b < 0 || e > nnz;
+  if (!bad) {
+    for (int p = b + lane; p < e; p += 32) {
+      const int32_t j = kv_idx[p];
+      if (j < 0 || j >= nKb) bad = true;
+      if (p > b && kv_idx[p - 1] >= j) bad = true;
+    }
+  }
+  if (bad) report_error(status, LOSA_ERR_BAD_INDEX);
+}
+
+int next_pow2(int x) {
+  int n = 32;
+  while (n < x) n <<= 1;
+  return n;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+size_t select_workspace_bytes(int64_t rows, int nKb) {
+  const size_t words = (size_t)(nKb + 31) / 32;
+  return align_up((size_t)rows * sizeof(int32_t), 256) + (size_t)rows * words * sizeof(uint32_t);
+}
+
+int launch_select(int rows, int nKb, const float* mass, double tau, int32_t* offsets,
+                  int32_t* kv_idx, int64_t kv_capacity, void* ws, cudaStream_t st) {
+  int* status = status_word_device();
+  if (!status) return LOSA_ERR_CUDA;
+  int32_t* counts = static_cast<int32_t*>(ws);
+  uint32_t* bitmaps = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) +
+                                                  align_up((size_t)rows * sizeof(int32_t), 256));
+  const int n2 = next_pow2(nKb);
+  const int words = (nKb + 31) / 32;
+  const size_t smem = (size_t)n2 * 8 + (size_t)words * 4;
+  if (smem > 48 * 1024) {
+    LOSA_CUDA_TRY(cudaFuncSetAttribute(select_rows_kernel,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  }
+  select_rows_kernel<<<rows, kSelThreads, smem, st>>>(mass, nKb, n2, tau, counts, bitmaps, status);
+  scan_counts_kernel<<<1, 1024, 0, st>>>(counts, rows, offsets, kv_capacity, status);
+  const int warps_per_cta = 8;
+  expand_rows_kernel<<<(rows + warps_per_cta - 1) / warps_per_cta, warps_per_cta * 32, 0, st>>>(
+      bitmaps, offsets, rows, nKb, kv_idx, kv_capacity);
+  LOSA_CUDA_TRY(cudaGetLastError());
+  return LOSA_OK;
+}
+
+int launch_validate_csr(int rows, int nKb, const int32_t* offsets, const int32_t* kv_idx,
+                        cudaStream_t st) {
+  int* status = status_word_device();
+  if (!status) return LOSA_ERR_CUDA;
+  validate_csr_kernel<<<(rows + 7) / 8, 256, 0, st>>>(rows, nKb, offsets, kv_idx, status);
+  LOSA_CUDA_TRY(cudaGetLastError());
+  return LOSA_OK;
+}
+
+}  // namespace losa

@@ -1,0 +1,199 @@
+"""Dense attention, block-sparse attention and the block-mass pass on the GPU against the fp64
+oracle, element by element, through the C ABI.  Sizes span several tiles, odd tile counts, both
+block geometries and ragged tails."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import losa_oracle as orc
+from paper_2608_12032_b200 import inputs
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+# (B, H, N, D, BLK): several 128-row tiles, odd numbers of tiles, short last blocks
+SHAPES = [
+    (1, 1, 128, 128, 128),
+    (1, 2, 256, 64, 64),
+    (1, 2, 300, 128, 128),
+    (2, 2, 1000, 64, 64),
+    (1, 3, 777, 128, 64),
+    (1, 2, 650, 64, 128),
+    (1, 1, 1500, 128, 128),
+]
+
+
+def lib():
+    import paper_2608_12032_b200 as losa
+    return losa
+
+
+def make(B, H, N, D, seed, scale=1.0):
+    return tuple(util.rand_bf16((B, H, N, D), seed + i, scale) for i in range(3))
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_dense_attention_matches_oracle(shape, out_dtype):
+    losa = lib()
+    B, H, N, D, BLK = shape
+    q, k, v = make(B, H, N, D, 11, 1.5)
+    o = losa.losa_attn(q.cuda(), k.cuda(), v.cuda(), BLK, BLK, out_dtype=out_dtype)
+    assert losa.losa_async_status() == 0
+    ref = orc.dense_attn(util.to_np(q), util.to_np(k), util.to_np(v))
+    if out_dtype == torch.bfloat16:
+        # compare with the oracle rounded to the output type as well as raw
+        ref_r = torch.from_numpy(ref).bfloat16().double().numpy()
+        assert np.abs(util.to_np(o) - ref_r).max() <= util.MAX_ABS_TOL
+    util.assert_output_close(o, ref, f"dense {shape}")
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("keep_prob", [0.15, 0.6])
+def test_sparse_attention_matches_oracle_on_random_patterns(shape, keep_prob):
+    losa = lib()
+    B, H, N, D, BLK = shape
+    q, k, v = make(B, H, N, D, 21, 1.5)
+    nQb = nKb = -(-N // BLK)
+    off, idx = util.random_csr(B * H * nQb, nKb, 5 + N, keep_prob)
+    o = losa.losa_sparse_attn(q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(off).cuda(),
+                              torch.from_numpy(idx).cuda(), BLK, BLK, out_dtype=torch.float32)
+    assert losa.losa_async_status() == 0
+    ref = orc.blocks_to_tokens(
+        orc.sparse_attn(util.to_np(q), util.to_np(k), util.to_np(v), BLK, BLK, off, idx), B, H, N)
+    util.assert_output_close(o, ref, f"sparse {shape}")
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+def test_sparse_with_all_blocks_equals_own_dense(shape):
+    losa = lib()
+    B, H, N, D, BLK = shape
+    q, k, v = (t.cuda() for t in make(B, H, N, D, 31))
+    nb = -(-N // BLK)
+    off, idx = util.all_blocks_csr(B * H * nb, nb)
+    o_s = losa.losa_sparse_attn(q, k, v, torch.from_numpy(off).cuda(), torch.from_numpy(idx).cuda(),
+                                BLK, BLK, out_dtype=torch.float32)
+    o_d = losa.losa_attn(q, k, v, BLK, BLK, out_dtype=torch.float32)
+    assert losa.losa_async_status() == 0
+    assert torch.equal(o_s, o_d)  # same tiles in the same order: bit-identical
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+def test_block_mass_matches_oracle(shape):
+    losa = lib()
+    B, H, N, D, BLK = shape
+    q, k, _ = make(B, H, N, D, 41, 1.5)
+    mass, lse = losa.losa_block_mass(q.cuda(), k.cuda(), BLK, BLK, return_lse=True)
+    assert losa.losa_async_status() == 0
+    ref, ref_lse = orc.block_mass(util.to_np(q), util.to_np(k), BLK, BLK, return_lse=True)
+    got = mass.cpu().numpy().reshape(ref.shape).astype(np.float64)
+    assert np.abs(got - ref).max() <= util.MASS_TOL
+    assert np.abs(got.sum(1) - 1.0).max() <= util.MASS_TOL
+    nQb = -(-N // BLK)
+    lse_ref = ref_lse.reshape(B, H, nQb * BLK)[:, :, :N]
+    assert np.abs(lse.cpu().numpy() - lse_ref).max() <= 1e-3
+
+
+@pytest.mark.parametrize("name,taus", [("tiny", (0.5, 0.75, 0.9, 0.99)), ("small", (0.9, 0.99, 1.0))])
+def test_chain_mass_select_sparse_on_named_workloads(name, taus):
+    """mass -> select -> sparse on the generator's tensors: strict selection parity on the GPU's
+    own masses, chain differences explained by the mass error, output parity on the oracle CSR."""
+    losa = lib()
+    wl = inputs.WORKLOADS[name]
+    q, k, v = inputs.make_qkv(wl, 0)
+    qn, kn, vn = (util.to_np(t) for t in (q, k, v))
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    mass = losa.losa_block_mass(qd, kd, wl.R, wl.C)
+    ref_mass = orc.block_mass(qn, kn, wl.R, wl.C)
+    gm = mass.cpu().numpy().reshape(ref_mass.shape)
+    mass_err = np.abs(gm - ref_mass).max()
+    assert mass_err <= util.MASS_TOL
+    for tau in taus:
+        off, idx = losa.losa_select(mass, tau)
+        assert losa.losa_async_status() == 0
+        off_h, idx_h = off.cpu().numpy(), idx.cpu().numpy()
+        # strict: the oracle's rule on the very same fp32 masses
+        strict = orc.select(gm.astype(np.float64), tau)
+        bad, _ = util.compare_csr(off_h, idx_h, strict)
+        assert not bad
+        # chain: oracle masses -> oracle selection; differences only where the decision was
+        # closer to tau than the mass error allows
+        chain = orc.select(ref_mass, tau)
+        mine, ref = util.csr_rows(off_h, idx_h[: off_h[-1]]), util.csr_rows(chain.offsets, chain.kv_idx)
+        dist = chain.boundary_distance()
+        for r, (a, b) in enumerate(zip(mine, ref)):
+            if a != b:
+                assert dist[r] <= mass_err * wl.nKb + util.NEAR_TAU
+        # output parity with the same CSR on both sides (the oracle's)
+        o = losa.losa_sparse_attn(qd, kd, vd, torch.from_numpy(chain.offsets).cuda(),
+                                  torch.from_numpy(chain.kv_idx).cuda(), wl.R, wl.C,
+                                  out_dtype=torch.float32)
+        ref_o = orc.blocks_to_tokens(
+            orc.sparse_attn(qn, kn, vn, wl.R, wl.C, chain.offsets, chain.kv_idx), wl.B, wl.H, wl.N)
+        util.assert_output_close(o, ref_o, f"{name} tau={tau}")
+        assert orc.recall(ref_mass, off_h, idx_h[: off_h[-1]]) >= tau - 1e-4
+    assert losa.losa_async_status() == 0
+
+
+def test_strided_heads_layout():
+    """[B, N, H, D] storage viewed as [B, H, N, D]: strides come from the problem description."""
+    losa = lib()
+    B, H, N, D, BLK = 1, 3, 400, 64, 64
+    base = [util.rand_bf16((B, N, H, D), 51 + i) for i in range(3)]
+    q, k, v = (t.cuda().permute(0, 2, 1, 3) for t in base)
+    assert not q.is_contiguous()
+    o = losa.losa_attn(q, k, v, BLK, BLK, out_dtype=torch.float32)
+    assert losa.losa_async_status() == 0 and o.stride() == q.stride()
+    qn, kn, vn = (util.to_np(t.permute(0, 2, 1, 3)) for t in base)
+    util.assert_output_close(o, orc.dense_attn(qn, kn, vn), "strided")
+
+
+def test_bad_block_index_is_reported_and_skipped():
+    losa = lib()
+    B, H, N, D, BLK = 1, 1, 512, 64, 64
+    q, k, v = (t.cuda() for t in make(B, H, N, D, 61))
+    off, idx = util.random_csr(8, 8, 1, 0.5)
+    good = idx.copy()
+    bad = idx.copy()
+    victim = int(off[3])
+    bad[victim] = 99  # out of range: must be skipped, not dereferenced
+    o = losa.losa_sparse_attn(q, k, v, torch.from_numpy(off).cuda(), torch.from_numpy(bad).cuda(),
+                              BLK, BLK, out_dtype=torch.float32)
+    assert losa.losa_status_string(losa.losa_async_status()) == "LOSA_ERR_BAD_INDEX"
+    assert torch.isfinite(o).all()
+    # the other rows are unaffected
+    o_good = losa.losa_sparse_attn(q, k, v, torch.from_numpy(off).cuda(),
+                                   torch.from_numpy(good).cuda(), BLK, BLK, out_dtype=torch.float32)
+    assert losa.losa_async_status() == 0
+    keep = torch.ones(N, dtype=torch.bool)
+    keep[3 * BLK:4 * BLK] = False
+    assert torch.equal(o[0, 0, keep.cuda()], o_good[0, 0, keep.cuda()])
+
+
+def test_host_side_argument_errors():
+    losa = lib()
+    q = torch.zeros(1, 1, 128, 96, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(losa.LosaError) as e:
+        losa.losa_attn(q, q, q, 128, 128)
+    assert e.value.code == -2
+    q = torch.zeros(1, 1, 128, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(losa.LosaError) as e:
+        losa.losa_attn(q, q, q, 128, 32)
+    assert e.value.code == -2
+    with pytest.raises(losa.LosaError) as e:
+        losa.losa_block_mass(q, q, 64, 64, ws=torch.empty(64, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == -3
+
+
+def test_kernels_are_deterministic():
+    losa = lib()
+    wl = dataclasses.replace(inputs.WORKLOADS["small"], H=2)
+    q, k, v = (t.cuda() for t in inputs.make_qkv(wl, 3))
+    m1 = losa.losa_block_mass(q, k, wl.R, wl.C)
+    m2 = losa.losa_block_mass(q, k, wl.R, wl.C)
+    o1 = losa.losa_attn(q, k, v, wl.R, wl.C)
+    o2 = losa.losa_attn(q, k, v, wl.R, wl.C)
+    assert losa.losa_async_status() == 0
+    assert torch.equal(m1, m2) and torch.equal(o1, o2)

@@ -1,0 +1,123 @@
+"""losa_select and losa_validate_csr on the GPU against the oracle's Eq. 3, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import losa_oracle as orc
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+def lib():
+    import paper_2608_12032_b200 as losa
+    return losa
+
+
+def random_mass(rows, nKb, seed, tail=3.0):
+    rng = np.random.default_rng(seed)
+    m = np.exp(tail * rng.standard_normal((rows, nKb)))
+    return (m / m.sum(1, keepdims=True)).astype(np.float32)
+
+
+def run_select(m32, tau, B=1, H=1, **kw):
+    losa = lib()
+    rows, nKb = m32.shape
+    mass = torch.from_numpy(m32).cuda().reshape(B, H, rows // (B * H), nKb)
+    off, idx = losa.losa_select(mass, tau, **kw)
+    status = losa.losa_async_status()
+    return off.cpu().numpy(), idx.cpu().numpy(), status
+
+
+@pytest.mark.parametrize("rows,nKb", [(8, 1), (8, 4), (64, 31), (64, 32), (64, 33), (96, 256),
+                                      (40, 278), (24, 929), (6, 1500), (3, 5000)])
+@pytest.mark.parametrize("tau", [0.5, 0.99, 1.0])
+def test_select_bit_exact_against_oracle(rows, nKb, tau):
+    m32 = random_mass(rows, nKb, 1000 + nKb)
+    off, idx, status = run_select(m32, tau)
+    assert status == 0
+    sel = orc.select(m32.astype(np.float64), tau)
+    bad, exempt = util.compare_csr(off, idx, sel)
+    assert not bad, f"rows {bad[:5]} differ"
+    assert exempt == 0 or tau < 1.0
+    assert off[0] == 0 and off[-1] == sel.count.sum()
+
+
+def test_select_ties_uniform_and_zero_masses():
+    nKb = 10
+    m = np.full((4, nKb), 0.1, dtype=np.float32)
+    off, idx, status = run_select(m, 0.75)
+    sel = orc.select(m.astype(np.float64), 0.75)
+    assert status == 0 and not util.compare_csr(off, idx, sel)[0]
+    assert list(idx[: off[1]]) == list(range(sel.count[0]))
+    m = np.array([[0.1, 0.3, 0.3, 0.1, 0.2], [0.0, 0.0, 1.0, 0.0, -0.0]], dtype=np.float32)
+    for tau in (0.55, 0.85, 0.99):
+        off, idx, status = run_select(m, tau)
+        sel = orc.select(np.abs(m).astype(np.float64), tau)
+        assert status == 0 and not util.compare_csr(off, idx, sel)[0]
+
+
+def test_select_is_deterministic_and_multi_head():
+    m32 = random_mass(2 * 3 * 16, 70, 5)
+    a = run_select(m32, 0.9, B=2, H=3)
+    b = run_select(m32, 0.9, B=2, H=3)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1][: a[0][-1]], b[1][: b[0][-1]])
+    sel = orc.select(m32.astype(np.float64), 0.9)
+    assert not util.compare_csr(a[0], a[1], sel)[0]
+
+
+def test_select_reports_capacity_overflow_without_writing_past_it():
+    losa = lib()
+    m32 = random_mass(16, 64, 7)
+    sel = orc.select(m32.astype(np.float64), 0.99)
+    nnz = int(sel.count.sum())
+    cap = nnz // 2
+    mass = torch.from_numpy(m32).cuda().reshape(1, 1, 16, 64)
+    offsets = torch.empty(17, dtype=torch.int32, device="cuda")
+    kv = torch.full((nnz,), -7, dtype=torch.int32, device="cuda")
+    losa.losa_select(mass, 0.99, kv_capacity=cap, out=(offsets, kv))
+    assert losa.losa_status_string(losa.losa_async_status()) == "LOSA_ERR_CAPACITY"
+    assert int(offsets[-1]) == nnz  # offsets stay exact
+    assert torch.all(kv[cap:] == -7)
+    assert np.array_equal(kv[:cap].cpu().numpy(), sel.kv_idx[:cap])
+    assert losa.losa_async_status() == 0  # the status word was cleared
+
+
+def test_select_flags_negative_and_nan_mass():
+    losa = lib()
+    m = random_mass(4, 16, 9)
+    m[1, 3] = -0.5
+    m[2, 5] = np.nan
+    run = run_select(m, 0.9)
+    assert losa.losa_status_string(run[2]) == "LOSA_ERR_BAD_MASS"
+
+
+def test_select_host_side_argument_errors():
+    losa = lib()
+    mass = torch.rand(1, 1, 4, 8, device="cuda")
+    for tau in (0.0, -1.0, 1.5, float("nan")):
+        with pytest.raises(losa.LosaError) as e:
+            losa.losa_select(mass, tau)
+        assert e.value.code == -1
+    with pytest.raises(losa.LosaError) as e:
+        losa.losa_select(mass, 0.9, ws=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == -3
+
+
+def test_validate_csr():
+    losa = lib()
+    off, idx = util.random_csr(50, 40, 3)
+    o, i = torch.from_numpy(off).cuda(), torch.from_numpy(idx).cuda()
+    losa.losa_validate_csr(o, i, 40)
+    assert losa.losa_async_status() == 0
+    for mutate in ("range", "order", "empty"):
+        off2, idx2 = off.copy(), idx.copy()
+        if mutate == "range":
+            idx2[off2[7]] = 40
+        elif mutate == "order":
+            r = int(np.argmax(np.diff(off2) >= 2))
+            idx2[off2[r]], idx2[off2[r] + 1] = idx2[off2[r] + 1], idx2[off2[r]]
+        else:
+            off2[10] = off2[11]
+        losa.losa_validate_csr(torch.from_numpy(off2).cuda(), torch.from_numpy(idx2).cuda(), 40)
+        assert losa.losa_status_string(losa.losa_async_status()) == "LOSA_ERR_BAD_INDEX", mutate
