@@ -1,0 +1,441 @@
+#!/usr/bin/env python
+"""Benchmark of LoSA's attention hot path on B200.
+
+One "step" is one pass of the whole path over one synthetic attention layer:
+
+    losa_block_mass(q0, k0) -> losa_select(mass, tau)           (one-time construction)
+    losa_sparse_attn(q_t, k_t, v_t, CSR) for t = 1..draws        (frozen pattern, later steps)
+    losa_attn(q_1, k_1, v_1)                                     (own dense forward, for the ratio)
+
+The headline value is the effective TFLOP/s of the block-sparse forward, counting the flops of
+the retained blocks only.  Everything is timed with CUDA events on the launching stream.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload wan] [--draws 10]
+    python bench.py --impl reference ...      # the fp64 CPU oracle on a bounded sample
+
+Under torchrun every rank runs the same layer shape on its own seeds (weak scaling; the path has
+no exchange step, so there is no data-path collective) and rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_2608_12032_b200 import inputs  # noqa: E402
+
+METRIC = "block_sparse_attn_effective_tflops"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="losa", choices=["losa", "reference"])
+    ap.add_argument("--workload", default="wan", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--draws", type=int, default=10, help="reuse draws per step")
+    ap.add_argument("--tau", type=float, default=None)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-baseline sample")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+def retained_flops(wl, offsets: np.ndarray, kv_idx: np.ndarray) -> float:
+    """4 * d * sum over retained (query block, key block) pairs of |B_i| * |B_j| (valid tokens)."""
+    nQb, nKb = wl.nQb, wl.nKb
+    qsz = np.full(nQb, wl.R, dtype=np.int64)
+    qsz[-1] = wl.N - (nQb - 1) * wl.R
+    ksz = np.full(nKb, wl.C, dtype=np.int64)
+    ksz[-1] = wl.N - (nKb - 1) * wl.C
+    counts = np.diff(offsets.astype(np.int64))
+    row_q = np.tile(qsz, wl.B * wl.H)
+    per_entry_q = np.repeat(row_q, counts)
+    return 4.0 * wl.D * float((per_entry_q * ksz[kv_idx[: offsets[-1]]]).sum())
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.05)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {
+            "sm_mhz": statistics.median(self.samples) if self.samples else None,
+            "sm_max_mhz": self.max_mhz,
+            "reasons": sorted(self.reasons),
+            "samples": len(self.samples),
+        }
+
+
+def cpu_baseline(wl, q, k, v, offsets, kv_idx, seconds: float):
+    """The oracle's sparse attention (Eq. 4), as it stands, on a bounded sample of query blocks."""
+    from oracle import losa_oracle as orc
+
+    qn, kn, vn = (t.float().numpy() for t in (q, k, v))
+    rows = wl.rows
+    rng = np.random.default_rng(0)
+    order = rng.permutation(rows)
+    nQb = wl.nQb
+    done, flops, t0 = 0, 0.0, time.perf_counter()
+    chunk = max(1, orc.threads() // 16)
+    ksz = np.full(wl.nKb, wl.C, dtype=np.int64)
+    ksz[-1] = wl.N - (wl.nKb - 1) * wl.C
+    while done < rows:
+        ids = np.sort(order[done:done + chunk]).astype(np.int32)
+        orc.sparse_attn(qn, kn, vn, wl.R, wl.C, offsets, kv_idx, row_ids=ids)
+        for r in ids:
+            i = int(r) % nQb
+            qrows = min(wl.R, wl.N - i * wl.R)
+            flops += 4.0 * wl.D * qrows * float(ksz[kv_idx[offsets[r]:offsets[r + 1]]].sum())
+        done += len(ids)
+        if time.perf_counter() - t0 >= seconds:
+            break
+    dt = time.perf_counter() - t0
+    return {
+        "value": flops / dt / 1e12,
+        "unit": UNIT,
+        "cores": orc.threads(),
+        "kind": "oracle",
+        "sample": f"fp64 oracle sparse attention on {done} of {rows} query blocks "
+                  f"(random sample, seed 0) of the {wl.name} workload in {dt:.1f} s",
+        "seconds": dt,
+        "blocks": done,
+    }
+
+
+def run_reference(args, wl, rank, world):
+    """Reference arm: the fp64 CPU oracle, timed on this machine's host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    from oracle import losa_oracle as orc
+
+    tau = wl.tau if args.tau is None else args.tau
+    q, k, v = inputs.make_qkv(wl, 0)
+    qn, kn, vn = (t.float().numpy() for t in (q, k, v))
+    # the pattern of a bounded sample of query blocks, from the oracle's own masses
+    per_step = max(2, min(32, orc.threads()))
+    rng = np.random.default_rng(0)
+    total = args.warmup + args.steps
+    ids_all = rng.choice(wl.rows, size=min(wl.rows, per_step * total), replace=False).astype(np.int32)
+    times, flops = [], []
+    ksz = np.full(wl.nKb, wl.C, dtype=np.int64)
+    ksz[-1] = wl.N - (wl.nKb - 1) * wl.C
+    for s in range(total):
+        ids = np.sort(ids_all[s * per_step:(s + 1) * per_step])
+        if ids.size == 0:
+            ids = np.sort(ids_all[:per_step])
+        t0 = time.perf_counter()
+        mass = orc.block_mass(qn, kn, wl.R, wl.C, row_ids=ids)
+        sel = orc.select(mass, tau)
+        # CSR over all rows with only the sampled rows populated
+        counts = np.ones(wl.rows, dtype=np.int64)
+        counts[ids] = sel.count
+        off = np.zeros(wl.rows + 1, dtype=np.int64)
+        np.cumsum(counts, out=off[1:])
+        idx = np.zeros(off[-1], dtype=np.int32)
+        for n, r in enumerate(ids):
+            idx[off[r]:off[r + 1]] = sel.kept[n, : sel.count[n]]
+        t1 = time.perf_counter()
+        orc.sparse_attn(qn, kn, vn, wl.R, wl.C, off.astype(np.int32), idx, row_ids=ids)
+        t2 = time.perf_counter()
+        f = 0.0
+        for n, r in enumerate(ids):
+            qrows = min(wl.R, wl.N - (int(r) % wl.nQb) * wl.R)
+            f += 4.0 * wl.D * qrows * float(ksz[sel.kept[n, : sel.count[n]]].sum())
+        if s >= args.warmup:
+            times.append((t2 - t0, t2 - t1))
+            flops.append(f)
+    sparse_s = sum(t[1] for t in times)
+    value = sum(flops) / sparse_s / 1e12
+    line = {
+        "impl": "reference",
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * sum(t[0] for t in times) / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "tau": tau, "sample_blocks_per_step": per_step,
+                   "note": "each step = oracle mass + select + sparse attention on a sample of query blocks"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.threads(), "kind": "oracle",
+                         "sample": f"{per_step} random query blocks of {wl.rows} per step"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    wl = inputs.WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, wl, rank, world)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    import paper_2608_12032_b200 as losa
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=dev)
+
+    tau = wl.tau if args.tau is None else args.tau
+    base_seed = 1000 * rank  # rank r draws its own layer
+    peaks = load_peaks()
+
+    # ---- inputs: step-0 tensors and the reuse draws, resident in HBM before timing starts
+    base = inputs.make_base_fp32(wl, base_seed)
+    q0, k0, v0 = (t.bfloat16() for t in base)
+    host_draws = [inputs.make_reuse_draw(wl, base_seed + t, base=base) for t in range(1, args.draws + 1)]
+    del base
+    q0d, k0d = q0.to(dev), k0.to(dev)
+    draws = [tuple(t.to(dev) for t in d) for d in host_draws]
+
+    prob = losa.make_problem(q0d, wl.R, wl.C)
+    rows, nKb = wl.rows, wl.nKb
+    ws_mass = torch.empty(losa.losa_workspace_bytes(0, prob), dtype=torch.uint8, device=dev)
+    mass = torch.empty((wl.B, wl.H, wl.nQb, nKb), dtype=torch.float32, device=dev)
+    offsets = torch.empty(rows + 1, dtype=torch.int32, device=dev)
+    kv_idx = torch.empty(rows * nKb, dtype=torch.int32, device=dev)
+    ws_sel = torch.empty(max(1, losa.binding._select_workspace_bytes(wl.B, wl.H, wl.nQb, nKb)),
+                         dtype=torch.uint8, device=dev)
+    o_sparse = torch.empty_like(draws[0][0])
+    o_dense = torch.empty_like(draws[0][0])
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def step(record=None):
+        marks = [ev()]
+        marks[0].record()
+        losa.losa_block_mass(q0d, k0d, wl.R, wl.C, ws=ws_mass, mass=mass)
+        marks.append(ev()); marks[-1].record()
+        losa.losa_select(mass, tau, ws=ws_sel, out=(offsets, kv_idx))
+        marks.append(ev()); marks[-1].record()
+        for (q, k, v) in draws:
+            losa.losa_sparse_attn(q, k, v, offsets, kv_idx, wl.R, wl.C, out=o_sparse)
+            marks.append(ev()); marks[-1].record()
+        q, k, v = draws[0]
+        losa.losa_attn(q, k, v, wl.R, wl.C, out=o_dense)
+        marks.append(ev()); marks[-1].record()
+        if record is not None:
+            record.append(marks)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    losa.check_async("warm-up")
+    off_h = offsets.cpu().numpy()
+    idx_h = kv_idx[: int(off_h[-1])].cpu().numpy()
+    flops_sparse = retained_flops(wl, off_h, idx_h)
+    coverage = float(off_h[-1]) / float(rows * nKb)
+
+    records = []
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        t_start, t_end = ev(), ev()
+        t_start.record()
+        for _ in range(args.steps):
+            step(records)
+        t_end.record()
+        barrier()
+    losa.check_async("timed region")
+    total_ms = t_start.elapsed_time(t_end)
+
+    mass_ms, sel_ms, sparse_ms, dense_ms = [], [], [], []
+    for marks in records:
+        mass_ms.append(marks[0].elapsed_time(marks[1]))
+        sel_ms.append(marks[1].elapsed_time(marks[2]))
+        for i in range(args.draws):
+            sparse_ms.append(marks[2 + i].elapsed_time(marks[3 + i]))
+        dense_ms.append(marks[2 + args.draws].elapsed_time(marks[3 + args.draws]))
+    sparse_total_ms = sum(sparse_ms)
+
+    # max over ranks of the times that enter the aggregate
+    t = torch.tensor([total_ms, sparse_total_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms_max, sparse_total_ms_max = (float(x) for x in t.cpu())
+    n_sparse_calls = args.steps * args.draws
+    value = world * flops_sparse * n_sparse_calls / (sparse_total_ms_max * 1e-3) / 1e12
+
+    # ---- end to end through the public API with host buffers (pinned), copies inside the timing
+    e2e = None
+    if not args.no_e2e:
+        pin = [tuple(t.pin_memory() for t in d) for d in host_draws]
+        q0p, k0p = q0.pin_memory(), k0.pin_memory()
+        o_host = torch.empty(o_sparse.shape, dtype=o_sparse.dtype).pin_memory()
+        qd, kd, vd = (torch.empty_like(draws[0][0]) for _ in range(3))
+
+        def e2e_step():
+            qd.copy_(q0p, non_blocking=True)
+            kd.copy_(k0p, non_blocking=True)
+            losa.losa_block_mass(qd, kd, wl.R, wl.C, ws=ws_mass, mass=mass)
+            losa.losa_select(mass, tau, ws=ws_sel, out=(offsets, kv_idx))
+            for (q, k, v) in pin:
+                qd.copy_(q, non_blocking=True)
+                kd.copy_(k, non_blocking=True)
+                vd.copy_(v, non_blocking=True)
+                losa.losa_sparse_attn(qd, kd, vd, offsets, kv_idx, wl.R, wl.C, out=o_sparse)
+                o_host.copy_(o_sparse, non_blocking=True)
+
+        e2e_step()
+        barrier()
+        a, b = ev(), ev()
+        n_e2e = max(1, min(args.steps, 2))
+        a.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        b.record()
+        barrier()
+        e2e_ms = torch.tensor([a.elapsed_time(b)], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+        nbytes = q0.numel() * 2
+        e2e = {
+            "value": world * flops_sparse * args.draws * n_e2e / (float(e2e_ms) * 1e-3) / 1e12,
+            "unit": UNIT,
+            "h2d_bytes_per_step": (2 + 3 * args.draws) * nbytes,
+            "d2h_bytes_per_step": args.draws * nbytes,
+            "ms_per_step": float(e2e_ms) / n_e2e,
+            "steps": n_e2e,
+            "note": "mass+select+draws x sparse attention; every call's q/k/v copied from pinned "
+                    "host memory and every output copied back inside the timed region",
+        }
+        losa.check_async("e2e")
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    sparse_avg_ms = sparse_total_ms / n_sparse_calls
+    achieved = flops_sparse / (sparse_avg_ms * 1e-3) / 1e12
+    peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+    dense_flops = wl.dense_flop()
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total_ms_max / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {
+            "workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "D": wl.D, "R": wl.R, "C": wl.C,
+            "tau": tau, "draws": args.draws, "coverage": coverage, "nnz": int(off_h[-1]),
+            "step": "block_mass + select + draws x sparse_attn + 1 dense attn",
+            "l2": "inputs larger than L2: each sparse call reads a different 300 MB draw",
+            "pe_base": wl.pe_base, "pe_scale": wl.pe_scale,
+        },
+        "ms_per_layer": {
+            "sparse_attn": sparse_avg_ms, "sparse_attn_min": min(sparse_ms),
+            "dense_attn": statistics.mean(dense_ms), "block_mass": statistics.mean(mass_ms),
+            "select": statistics.mean(sel_ms),
+        },
+        "sparse_vs_dense_speedup": statistics.mean(dense_ms) / sparse_avg_ms,
+        "dense_tflops": dense_flops / (statistics.mean(dense_ms) * 1e-3) / 1e12,
+        "block_mass_tflops": 0.5 * dense_flops / (statistics.mean(mass_ms) * 1e-3) / 1e12,
+        "roofline": {
+            "kernel": "losa_attn_kernel<sparse>", "bound": "tensor", "achieved": achieved,
+            "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+            "peak_source": f"{peaks['_source']} bf16_tflops_sustained (kernel timed inside a long step)",
+            "frac_of_burst": achieved / float(peaks["bf16_tflops"]),
+            "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS,
+            "flops_per_launch": flops_sparse,
+            "traffic": None,
+        },
+        "clocks": clocks.summary(),
+        "gpu_launches": args.steps * (1 + 3 + args.draws + 1),
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(wl, *host_draws[0], off_h, idx_h, args.cpu_seconds)
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

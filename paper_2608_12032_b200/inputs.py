@@ -129,16 +129,23 @@ def make_qkv(wl: Workload, seed: int = 0):
     return q.bfloat16(), k.bfloat16(), v.bfloat16()
 
 
-def make_reuse_draw(wl: Workload, draw: int, base_seed: int = 0, noise: float = 0.05):
+def make_base_fp32(wl: Workload, seed: int = 0):
+    """The fp32 tensors before the bf16 cast (what the reuse draws perturb)."""
+    return _base_fp32(wl, seed)
+
+
+def make_reuse_draw(wl: Workload, draw: int, base_seed: int = 0, noise: float = 0.05, base=None):
     """Later-step tensors: the step-0 fp32 tensors perturbed by `noise` * rms Gaussian noise.
 
     Stands in for the later denoising steps on which the frozen pattern is
     reused (the paper recomputes Q/K/V from the current hidden states at each
-    step and keeps the block indices fixed).
+    step and keeps the block indices fixed).  `base` may carry the result of
+    make_base_fp32(wl, base_seed) to avoid drawing it again.
     """
     if draw < 1:
         raise ValueError("reuse draws are numbered from 1")
-    base = _base_fp32(wl, base_seed)
+    if base is None:
+        base = _base_fp32(wl, base_seed)
     g = torch.Generator("cpu").manual_seed(draw)
     out = []
     for x in base:

@@ -1,0 +1,133 @@
+"""Parity at the benchmark's full sizes (CogVideoX-, Wan2.1- and HunyuanVideo-shaped layers), in
+the launch configuration bench.py times.  The GPU computes every row; the fp64 oracle computes a
+seeded sample of query blocks one by one (each query block depends only on its own queries and
+the head's full K/V, so a sampled block is verified exactly), and the selection rule is checked
+on every row."""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import losa_oracle as orc
+from paper_2608_12032_b200 import inputs
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+def sample_rows(wl, n, seed):
+    rng = np.random.default_rng(seed)
+    ids = set(rng.choice(wl.rows, size=n, replace=False).tolist())
+    ids.add(wl.nQb - 1)             # ragged last query block of the first head
+    ids.add(wl.rows - wl.nQb)       # first query block of the last head
+    return np.array(sorted(ids), dtype=np.int32)
+
+
+def gather_blocks(o: torch.Tensor, wl, ids):
+    """[B,H,N,D] device tensor -> [len(ids), R, D] numpy (rows >= N zero), like the oracle's layout."""
+    out = np.zeros((len(ids), wl.R, wl.D), dtype=np.float64)
+    flat = o.reshape(wl.B * wl.H, wl.N, wl.D)
+    for n, r in enumerate(ids):
+        bh, i = divmod(int(r), wl.nQb)
+        blk = flat[bh, i * wl.R:(i + 1) * wl.R].float().cpu().numpy()
+        out[n, : blk.shape[0]] = blk
+    return out
+
+
+def log(record):
+    path = os.environ.get("LOSA_PARITY_LOG")
+    if path:
+        with open(path, "a") as f:
+            f.write(json.dumps(record) + "\n")
+
+
+@pytest.mark.parametrize("name,n_sample", [("cogvideox", 10), ("wan", 8), ("hunyuan", 4)])
+def test_full_size_parity_on_sampled_query_blocks(name, n_sample):
+    import paper_2608_12032_b200 as losa
+
+    wl = inputs.WORKLOADS[name]
+    base = inputs.make_base_fp32(wl, 0)
+    q, k, v = (t.bfloat16() for t in base)
+    qn, kn, vn = (t.float().numpy() for t in (q, k, v))
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    ids = sample_rows(wl, n_sample, 7)
+
+    # ---- block mass (Eq. 1)
+    mass = losa.losa_block_mass(qd, kd, wl.R, wl.C)
+    losa.check_async("mass")
+    gm = mass.cpu().numpy().reshape(wl.rows, wl.nKb)
+    ref_mass = orc.block_mass(qn, kn, wl.R, wl.C, row_ids=ids)
+    mass_err = float(np.abs(gm[ids] - ref_mass).max())
+    assert mass_err <= util.MASS_TOL
+    assert np.abs(gm.astype(np.float64).sum(1) - 1.0).max() <= util.MASS_TOL  # every row, any size
+
+    # ---- selection (Eq. 3): every row, bit-exact on the GPU's own masses
+    off, idx = losa.losa_select(mass, wl.tau)
+    losa.losa_validate_csr(off, idx, wl.nKb)
+    losa.check_async("select")
+    off_h, idx_h = off.cpu().numpy(), idx.cpu().numpy()
+    strict = orc.select(gm.astype(np.float64), wl.tau)
+    bad, exempt = util.compare_csr(off_h, idx_h, strict)
+    assert not bad
+    coverage = orc.coverage(off_h, wl.nKb)
+    # chain on the sampled rows: oracle mass -> oracle selection
+    chain = orc.select(ref_mass, wl.tau)
+    chain_diff = 0
+    dist = chain.boundary_distance()
+    for n, r in enumerate(ids):
+        mine = tuple(idx_h[off_h[r]:off_h[r + 1]].tolist())
+        ref = tuple(chain.kept[n, : chain.count[n]].tolist())
+        if mine != ref:
+            chain_diff += 1
+            assert dist[n] <= mass_err * wl.nKb + util.NEAR_TAU
+
+    # ---- block-sparse forward (Eq. 4) with the same CSR on both sides
+    o = losa.losa_sparse_attn(qd, kd, vd, off, idx, wl.R, wl.C, out_dtype=torch.float32)
+    losa.check_async("sparse")
+    ref_o = orc.sparse_attn(qn, kn, vn, wl.R, wl.C, off_h, idx_h[: off_h[-1]], row_ids=ids)
+    d = np.abs(gather_blocks(o, wl, ids) - ref_o)
+    assert d.max() <= util.MAX_ABS_TOL and d.mean() <= util.MEAN_ABS_TOL
+    sparse_err = (float(d.max()), float(d.mean()))
+    del o
+
+    # ---- own dense forward on the same sampled blocks
+    o = losa.losa_attn(qd, kd, vd, wl.R, wl.C, out_dtype=torch.float32)
+    losa.check_async("dense")
+    counts = np.ones(wl.rows, dtype=np.int64)
+    counts[ids] = wl.nKb
+    doff = np.zeros(wl.rows + 1, dtype=np.int64)
+    np.cumsum(counts, out=doff[1:])
+    didx = np.zeros(doff[-1], dtype=np.int32)
+    for r in ids:
+        didx[doff[r]:doff[r + 1]] = np.arange(wl.nKb)
+    ref_d = orc.sparse_attn(qn, kn, vn, wl.R, wl.C, doff.astype(np.int32), didx, row_ids=ids)
+    d = np.abs(gather_blocks(o, wl, ids) - ref_d)
+    assert d.max() <= util.MAX_ABS_TOL and d.mean() <= util.MEAN_ABS_TOL
+    dense_err = (float(d.max()), float(d.mean()))
+    del o
+
+    record = {"workload": name, "sampled_blocks": len(ids), "rows": wl.rows, "coverage": coverage,
+              "nnz": int(off_h[-1]), "mass_max_abs": mass_err, "csr_mismatch_rows": len(bad),
+              "near_tau_exempt_rows": exempt, "chain_diff_rows_in_sample": chain_diff,
+              "sparse_max_abs": sparse_err[0], "sparse_mean_abs": sparse_err[1],
+              "dense_max_abs": dense_err[0], "dense_mean_abs": dense_err[1]}
+
+    # ---- the frozen pattern on a later draw (Wan protocol: indices reused on perturbed Q/K/V)
+    if name == "wan":
+        q1, k1, v1 = inputs.make_reuse_draw(wl, 1, base=base)
+        o = losa.losa_sparse_attn(q1.cuda(), k1.cuda(), v1.cuda(), off, idx, wl.R, wl.C,
+                                  out_dtype=torch.float32)
+        losa.check_async("sparse on reuse draw")
+        q1n, k1n, v1n = (t.float().numpy() for t in (q1, k1, v1))
+        ref_o = orc.sparse_attn(q1n, k1n, v1n, wl.R, wl.C, off_h, idx_h[: off_h[-1]], row_ids=ids)
+        d = np.abs(gather_blocks(o, wl, ids) - ref_o)
+        assert d.max() <= util.MAX_ABS_TOL and d.mean() <= util.MEAN_ABS_TOL
+        m1 = orc.block_mass(q1n, k1n, wl.R, wl.C, row_ids=ids)
+        kept = [m1[n, idx_h[off_h[r]:off_h[r + 1]]].sum() for n, r in enumerate(ids)]
+        record.update(reuse_draw_max_abs=float(d.max()), reuse_draw_mean_abs=float(d.mean()),
+                      reuse_draw_recall_min=float(min(kept)), reuse_draw_recall_mean=float(np.mean(kept)))
+        assert min(kept) >= 0.97  # frozen support keeps covering the mass on a perturbed step
+    log(record)
+    print(json.dumps(record))
