@@ -103,6 +103,39 @@ int losa_select(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const float* mas
                 int32_t* offsets, int32_t* kv_idx, int64_t kv_capacity, void* ws,
                 size_t ws_bytes, void* cuda_stream);
 
+/* Bytes of the scratch array built into the library for losa_select_noalloc (per GPU). */
+#define LOSA_SELECT_NOALLOC_MAX_SCRATCH (4u * 1024u * 1024u)
+
+/* losa_select for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this is a packaging variant of losa_select, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits or unaffordable - inside a
+ * latency-critical serving loop whose memory was carved up at start-up, under a framework
+ * whose allocator owns every byte of the device, or in a plugin that is handed its tensors
+ * and nothing else.  Such callers cannot supply the workspace losa_select asks for.  Here the
+ * workspace is a fixed array inside the library image instead: LOSA_SELECT_NOALLOC_MAX_SCRATCH
+ * bytes on every GPU that loads the library, held until the process exits.  The call performs
+ * no cudaMalloc, cudaFree, cudaHostAlloc or other allocating call, and unlike the other entry
+ * points it does not touch the library's pinned status word (creating that allocates).
+ *
+ * Same computation, arguments and results as losa_select, except:
+ *   - no workspace arguments.  The problem must fit the array: 256-byte-rounded 4*rows
+ *     plus 4*rows*ceil(nKb/32) bytes, plus 256, at most LOSA_SELECT_NOALLOC_MAX_SCRATCH
+ *     (all five benchmark shapes fit); otherwise LOSA_ERR_WORKSPACE is returned, nothing is
+ *     launched, and losa_last_cuda_error() says how many bytes were needed.
+ *   - device-side errors (LOSA_ERR_CAPACITY, LOSA_ERR_BAD_MASS) are not visible through
+ *     losa_async_status().  If device_status is not NULL it must point to an int32 in device
+ *     memory; the call writes LOSA_OK or the error code there, in stream order.
+ *   - the first call on each device looks up the array's device address (once per device,
+ *     with that device current).  Make that first call outside any stream capture.
+ *   - every call on a device shares the one array, which still holds the previous call's
+ *     contents.  The call clears what has to start at zero itself, so back-to-back calls on
+ *     one stream are fine; calls that can overlap on the GPU (different streams, different
+ *     host threads) race on the array and must be serialised by the caller. */
+int losa_select_noalloc(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const float* mass,
+                        double tau, int32_t* offsets, int32_t* kv_idx, int64_t kv_capacity,
+                        int32_t* device_status, void* cuda_stream);
+
 /* Block-sparse attention with a frozen pattern (Eq. 4).  Every valid query row q of query
  * block i attends to the valid keys of the blocks kv_idx[offsets[r] .. offsets[r+1]) only;
  * the softmax denominator runs over those keys only:

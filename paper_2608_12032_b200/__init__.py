@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     losa_attn,
     losa_block_mass,
     losa_select,
+    losa_select_noalloc,
     losa_sparse_attn,
     losa_status_string,
     losa_validate_csr,

@@ -21,7 +21,7 @@ LOSA_DTYPE_BF16, LOSA_DTYPE_F32 = 0, 1
 
 EXPORTS = (
     "losa_workspace_bytes", "losa_block_mass", "losa_select", "losa_sparse_attn", "losa_attn",
-    "losa_validate_csr", "losa_async_status", "losa_status_string", "losa_last_cuda_error",
+    "losa_select_noalloc", "losa_validate_csr", "losa_async_status", "losa_status_string", "losa_last_cuda_error",
 )
 
 
@@ -63,6 +63,8 @@ def _lib():
         lib.losa_block_mass.argtypes = [pp, vp, vp, vp, vp, vp, sz, vp]
         lib.losa_select.restype = ctypes.c_int
         lib.losa_select.argtypes = [i32, i32, i32, i32, vp, ctypes.c_double, vp, vp, i64, vp, sz, vp]
+        lib.losa_select_noalloc.restype = ctypes.c_int
+        lib.losa_select_noalloc.argtypes = [i32, i32, i32, i32, vp, ctypes.c_double, vp, vp, i64, vp, vp]
         lib.losa_sparse_attn.restype = ctypes.c_int
         lib.losa_sparse_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, ctypes.c_int, vp, sz, vp]
         lib.losa_attn.restype = ctypes.c_int
@@ -157,6 +159,23 @@ def losa_select(mass: torch.Tensor, tau: float, kv_capacity: Optional[int] = Non
     _check(_lib().losa_select(B, H, nQb, nKb, _ptr(mass), float(tau), _ptr(offsets), _ptr(kv_idx),
                               cap, _ptr(ws), ws.numel(), _stream()), "losa_select")
     return offsets, kv_idx
+
+
+def losa_select_noalloc(mass: torch.Tensor, tau: float, offsets: torch.Tensor, kv_idx: torch.Tensor,
+                        device_status: Optional[torch.Tensor] = None) -> None:
+    """losa_select without any allocation: for callers that own no allocator.
+
+    The caller passes every output (``offsets`` [rows + 1], ``kv_idx`` [capacity], optionally a
+    one-element int32 ``device_status``); the scratch memory is a fixed array inside the library.
+    This wrapper itself allocates nothing either.  Calls that may overlap on the GPU share that
+    array and must be serialised by the caller.
+    """
+    if mass.dim() != 4 or not mass.is_contiguous() or mass.dtype != torch.float32:
+        raise ValueError("mass must be a contiguous fp32 [B, H, nQb, nKb] tensor")
+    B, H, nQb, nKb = mass.shape
+    _check(_lib().losa_select_noalloc(B, H, nQb, nKb, _ptr(mass), float(tau), _ptr(offsets),
+                                      _ptr(kv_idx), kv_idx.numel(), _ptr(device_status), _stream()),
+           "losa_select_noalloc")
 
 
 def _select_workspace_bytes(B: int, H: int, nQb: int, nKb: int) -> int:

@@ -126,6 +126,26 @@ int losa_select(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const float* mas
                        static_cast<cudaStream_t>(cuda_stream));
 }
 
+int losa_select_noalloc(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const float* mass,
+                        double tau, int32_t* offsets, int32_t* kv_idx, int64_t kv_capacity,
+                        int32_t* device_status, void* cuda_stream) {
+  if (B <= 0 || H <= 0 || nQb <= 0 || nKb <= 0) return LOSA_ERR_INVALID_ARG;
+  if (!(tau > 0.0) || !(tau <= 1.0)) return LOSA_ERR_INVALID_ARG;
+  if (!mass || !offsets || !kv_idx || kv_capacity < 0) return LOSA_ERR_INVALID_ARG;
+  const int64_t rows = (int64_t)B * H * nQb;
+  if (rows * nKb > INT32_MAX || nKb > 8192) return LOSA_ERR_UNSUPPORTED;
+  const size_t need = select_workspace_bytes(rows, nKb);
+  if (need > select_noalloc_workspace_limit()) {
+    snprintf(g_cuda_error, sizeof(g_cuda_error),
+             "losa_select_noalloc: this mass matrix needs %zu bytes of scratch, the built-in "
+             "array holds %zu; use losa_select with caller-provided workspace",
+             need, select_noalloc_workspace_limit());
+    return LOSA_ERR_WORKSPACE;
+  }
+  return launch_select_noalloc((int)rows, nKb, mass, tau, offsets, kv_idx, kv_capacity,
+                               device_status, static_cast<cudaStream_t>(cuda_stream));
+}
+
 static int check_attn_args(const losa_problem_t* p, Geometry* g, const void* q, const void* k,
                            const void* v, const void* o, int o_dtype) {
   int rc = make_geometry(p, g);

@@ -233,6 +233,62 @@ int launch_select(int rows, int nKb, const float* mass, double tau, int32_t* off
   return LOSA_OK;
 }
 
+// ---- allocation-free variant ----------------------------------------------------------
+// Scratch for losa_select_noalloc lives in the library image: one array per GPU that loads
+// the library, held until the process exits.  The first 256 bytes hold the status word of
+// the last call, the rest is the counts + bitmaps workspace.
+constexpr size_t kStaticStatusBytes = 256;
+static __device__ __align__(256) unsigned char g_select_scratch[LOSA_SELECT_NOALLOC_MAX_SCRATCH];
+
+namespace {
+constexpr int kMaxDevices = 64;
+unsigned char* g_scratch_addr[kMaxDevices] = {};  // device address of g_select_scratch, per device
+}  // namespace
+
+size_t select_noalloc_workspace_limit() {
+  return (size_t)LOSA_SELECT_NOALLOC_MAX_SCRATCH - kStaticStatusBytes;
+}
+
+int launch_select_noalloc(int rows, int nKb, const float* mass, double tau, int32_t* offsets,
+                          int32_t* kv_idx, int64_t kv_capacity, int32_t* device_status,
+                          cudaStream_t st) {
+  int dev = 0;
+  LOSA_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return LOSA_ERR_UNSUPPORTED;
+  if (!g_scratch_addr[dev]) {
+    // In host code the array's name is only a handle; the device address must be asked for,
+    // once per device, with that device current.
+    unsigned char* ptr = nullptr;
+    LOSA_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_select_scratch));
+    g_scratch_addr[dev] = ptr;
+  }
+  unsigned char* base = g_scratch_addr[dev];
+  int* status = reinterpret_cast<int*>(base);
+  unsigned char* ws = base + kStaticStatusBytes;
+  // the array keeps the previous call's contents: the status word must start at zero; counts
+  // and bitmaps are fully rewritten by the first kernel before anything reads them
+  LOSA_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int), st));
+  int32_t* counts = reinterpret_cast<int32_t*>(ws);
+  uint32_t* bitmaps =
+      reinterpret_cast<uint32_t*>(ws + align_up((size_t)rows * sizeof(int32_t), 256));
+  const int n2 = next_pow2(nKb);
+  const int words = (nKb + 31) / 32;
+  const size_t smem = (size_t)n2 * 8 + (size_t)words * 4;
+  if (smem > 48 * 1024) {
+    LOSA_CUDA_TRY(cudaFuncSetAttribute(select_rows_kernel,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  }
+  select_rows_kernel<<<rows, kSelThreads, smem, st>>>(mass, nKb, n2, tau, counts, bitmaps, status);
+  scan_counts_kernel<<<1, 1024, 0, st>>>(counts, rows, offsets, kv_capacity, status);
+  const int warps_per_cta = 8;
+  expand_rows_kernel<<<(rows + warps_per_cta - 1) / warps_per_cta, warps_per_cta * 32, 0, st>>>(
+      bitmaps, offsets, rows, nKb, kv_idx, kv_capacity);
+  LOSA_CUDA_TRY(cudaGetLastError());
+  if (device_status)
+    LOSA_CUDA_TRY(cudaMemcpyAsync(device_status, status, sizeof(int), cudaMemcpyDeviceToDevice, st));
+  return LOSA_OK;
+}
+
 int launch_validate_csr(int rows, int nKb, const int32_t* offsets, const int32_t* kv_idx,
                         cudaStream_t st) {
   int* status = status_word_device();
