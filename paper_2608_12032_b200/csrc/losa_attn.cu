@@ -2,8 +2,9 @@
 // frozen CSR pattern (Eq. 4) and the exact block-mass pass (Eq. 1), as ONE warp-specialised
 // persistent kernel template.
 //
-// CTA = 10 warps.  Warps 0-3 and 4-7 are two softmax warpgroups, each owning one 128-row
-// query tile (thread = query row = TMEM lane).  Warp 8 (one elected thread) is the TMA
+// CTA = 12 warps.  Warps 0-3 and 4-7 are two softmax warpgroups, each owning one 128-row
+// query tile (thread = query row = TMEM lane); they take 216 registers per thread from the
+// third warpgroup (setmaxnreg), whose warps 10-11 idle.  Warp 8 (one elected thread) is the TMA
 // producer: it streams the query tiles and the K / V tiles named by the block indices into
 // 128B-swizzled shared-memory rings.  Warp 9 (one elected thread) issues the tcgen05 MMAs:
 // S = Q K^T from shared memory into TMEM, O += P V with P read from TMEM (bf16, aliasing S)
@@ -34,7 +35,13 @@
 namespace losa {
 namespace {
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;  // 2 softmax warpgroups + 1 utility warpgroup (TMA, MMA, 2 idle warps)
+constexpr int kRegsSoftmax = 216, kRegsUtility = 72, kRegsAtLaunch = 168;
+// setmaxnreg only moves registers inside the CTA's launch allocation: the increase waits until
+// the decrease has released enough, so the totals must balance or the increase never returns.
+static_assert(128 * kRegsUtility + 256 * kRegsSoftmax <= kThreads * kRegsAtLaunch,
+              "register reallocation exceeds the CTA's launch allocation");
+static_assert(kThreads * kRegsAtLaunch <= 65536, "launch allocation exceeds the register file");
 constexpr int kTmemCols = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -229,6 +236,10 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = ctl->tmem_base;
 
+  // The softmax warpgroups hold a whole S row per thread: the utility warpgroup (warps 8-11)
+  // gives registers up and the softmax warpgroups take them.
+  if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsUtility));
   if (warp == 8) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -380,8 +391,10 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
       }
     }
+  }
   } else {
     // ------------------------------------------------------------------ softmax warpgroups
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
     const int qt = warp >> 2, wl = warp & 3;
     const int row = wl * 32 + lane;
     const uint32_t lane_base = (uint32_t)(wl * 32) << 16;
@@ -417,21 +430,19 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
           for (int c0 = 0; c0 < kC; c0 += 32) ptx::tmem_ld32(tS + c0, &sr[c0]);
           ptx::tmem_wait_ld();
-          float s[kC];
-#pragma unroll
-          for (int c = 0; c < kC; ++c) s[c] = __uint_as_float(sr[c]);
           if (j == p.nKb - 1 && tail < kC) {
 #pragma unroll
             for (int c = 0; c < kC; ++c)
-              if (c >= tail) s[c] = -INFINITY;
+              if (c >= tail) sr[c] = 0xff800000u;  // -inf: the key does not exist
           }
-          float mx0 = s[0], mx1 = s[1], mx2 = s[2], mx3 = s[3];
+          float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
+          float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
 #pragma unroll
           for (int c = 4; c < kC; c += 4) {
-            mx0 = fmaxf(mx0, s[c]);
-            mx1 = fmaxf(mx1, s[c + 1]);
-            mx2 = fmaxf(mx2, s[c + 2]);
-            mx3 = fmaxf(mx3, s[c + 3]);
+            mx0 = fmaxf(mx0, __uint_as_float(sr[c]));
+            mx1 = fmaxf(mx1, __uint_as_float(sr[c + 1]));
+            mx2 = fmaxf(mx2, __uint_as_float(sr[c + 2]));
+            mx3 = fmaxf(mx3, __uint_as_float(sr[c + 3]));
           }
           const float m_new = fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
           const bool need = m_new > m_ref + kRescaleThreshold;
@@ -442,41 +453,46 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             if (C::kHasV && pv_item > 0) {
               LOSA_WAIT(&ctl->o_done[qt], (npv - 1) & 1);
               ptx::tc_fence_after_sync();
+              const float2 a2 = make_float2(alpha, alpha);
 #pragma unroll
               for (int c0 = 0; c0 < D; c0 += 32) {
                 uint32_t r[32];
                 ptx::tmem_ld32(tO + c0, r);
                 ptx::tmem_wait_ld();
 #pragma unroll
-                for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
+                for (int c = 0; c < 32; c += 2) {
+                  const float2 v = ptx::mul2(
+                      make_float2(__uint_as_float(r[c]), __uint_as_float(r[c + 1])), a2);
+                  r[c] = __float_as_uint(v.x);
+                  r[c + 1] = __float_as_uint(v.y);
+                }
                 ptx::tmem_st32(tO + c0, r);
               }
             }
           }
-          float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-          const float neg_m = -m_ref;
+          // p = 2^(s * scale_log2 - m_ref), two columns per instruction; the bf16 pair replaces
+          // the first of the two fp32 registers
+          const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+          const float2 nm2 = make_float2(-m_ref, -m_ref);
+          float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
 #pragma unroll
           for (int c = 0; c < kC; c += 4) {
-            s[c] = ptx::ex2_approx(fmaf(s[c], p.scale_log2, neg_m));
-            s[c + 1] = ptx::ex2_approx(fmaf(s[c + 1], p.scale_log2, neg_m));
-            s[c + 2] = ptx::ex2_approx(fmaf(s[c + 2], p.scale_log2, neg_m));
-            s[c + 3] = ptx::ex2_approx(fmaf(s[c + 3], p.scale_log2, neg_m));
-            l0 += s[c];
-            l1 += s[c + 1];
-            l2 += s[c + 2];
-            l3 += s[c + 3];
+            float2 x0 = ptx::fma2(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2);
+            float2 x1 = ptx::fma2(make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, nm2);
+            x0.x = ptx::ex2_approx(x0.x);
+            x0.y = ptx::ex2_approx(x0.y);
+            x1.x = ptx::ex2_approx(x1.x);
+            x1.y = ptx::ex2_approx(x1.y);
+            acc0 = ptx::add2(acc0, x0);
+            acc1 = ptx::add2(acc1, x1);
+            sr[c >> 1] = ptx::pack_bf16x2(x0.x, x0.y);
+            sr[(c >> 1) + 1] = ptx::pack_bf16x2(x1.x, x1.y);
           }
-          const float tsum = (l0 + l1) + (l2 + l3);
+          const float tsum = (acc0.x + acc0.y) + (acc1.x + acc1.y);
           l += tsum;
           if (C::kHasV) {
 #pragma unroll
-            for (int c0 = 0; c0 < kC / 2; c0 += 32) {
-              uint32_t pk[32];
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                pk[c] = ptx::pack_bf16x2(s[2 * (c0 + c)], s[2 * (c0 + c) + 1]);
-              ptx::tmem_st32(tS + c0, pk);
-            }
+            for (int c0 = 0; c0 < kC / 2; c0 += 32) ptx::tmem_st32(tS + c0, &sr[c0]);
           } else {
             tab[(int64_t)j * 128] = make_float2(tsum, m_ref);
           }
@@ -681,6 +697,13 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
   auto kern = losa_attn_kernel<D, BLK, MODE>;
   static bool configured = false;
   if (!configured) {
+    // the in-kernel register reallocation must fit the registers the CTA is launched with
+    cudaFuncAttributes attr;
+    LOSA_CUDA_TRY(cudaFuncGetAttributes(&attr, kern));
+    if (attr.numRegs * kThreads < 128 * kRegsUtility + 256 * kRegsSoftmax) {
+      set_cuda_error(cudaErrorLaunchOutOfResources, "register budget of losa_attn_kernel");
+      return LOSA_ERR_UNSUPPORTED;
+    }
     LOSA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     configured = true;
   }
