@@ -85,7 +85,7 @@ struct Control {
   uint64_t q_full[2], q_empty[2];
   uint64_t k_full[NK], k_empty[NK];
   uint64_t v_full[NV > 0 ? NV : 1], v_empty[NV > 0 ? NV : 1];
-  uint64_t s_full[2], p_ready[2], o_done[2], o_free[2];
+  uint64_t s_full[2], p_ready[2][2], o_done[2], o_free[2];  // p_ready: one per half of P
   uint64_t wg_bar[2];
   uint64_t drain;
   uint32_t tmem_base;
@@ -95,19 +95,29 @@ struct Control {
 
 // Ascending merge of the block-index lists of the (up to NB) query blocks of a work item.
 // Every role walks its own copy; the sequence is a pure function of the CSR, so they agree.
+// The whole warp walks it together: each lane keeps one entry of a 32-entry window per list
+// (one coalesced load per 32 tiles) and the current entry is broadcast with a shuffle, so no
+// role waits on a dependent global load per tile.  All 32 lanes must call every method.
 template <int NB>
 struct TileIter {
   const int32_t* idx;
-  int pos[NB], end[NB], cur[NB];
-  int nKb, dense_j;
+  int pos[NB], end[NB], cur[NB], base[NB], win[NB];
+  int nKb, dense_j, lane;
   uint32_t dense_mask;
   bool dense;
   int* status;
 
+  __device__ __forceinline__ void refill(int n) {
+    base[n] = pos[n];
+    const int at = pos[n] + lane;
+    win[n] = (at < end[n]) ? __ldg(idx + at) : INT_MAX;
+  }
+
   __device__ __forceinline__ void fetch(int n) {
     cur[n] = INT_MAX;
     while (pos[n] < end[n]) {
-      const int v = __ldg(idx + pos[n]);
+      if (pos[n] - base[n] >= 32) refill(n);
+      const int v = __shfl_sync(0xffffffffu, win[n], pos[n] - base[n]);
       if ((unsigned)v < (unsigned)nKb) {
         cur[n] = v;
         return;
@@ -117,19 +127,21 @@ struct TileIter {
     }
   }
 
-  __device__ __forceinline__ void init(const Params& p, bool is_dense, int bh, int first_block) {
+  __device__ __forceinline__ void init(const Params& p, bool is_dense, int bh, int first_block,
+                                       int lane_id) {
     idx = p.kv_idx;
     nKb = p.nKb;
     status = p.status;
     dense = is_dense;
     dense_j = 0;
     dense_mask = 0;
+    lane = lane_id;
     const int32_t nnz = is_dense ? 0 : __ldg(p.offsets + (int64_t)p.B * p.H * p.nQb);
 #pragma unroll
     for (int n = 0; n < NB; ++n) {
       const int g = first_block + n;
-      pos[n] = end[n] = 0;
-      cur[n] = INT_MAX;
+      pos[n] = end[n] = base[n] = 0;
+      cur[n] = win[n] = INT_MAX;
       if (g < p.nQb) {
         dense_mask |= 1u << n;
         if (!is_dense) {
@@ -140,6 +152,7 @@ struct TileIter {
           } else {
             pos[n] = b;
             end[n] = e;
+            refill(n);
             fetch(n);
           }
         }
@@ -171,6 +184,29 @@ struct TileIter {
     return true;
   }
 };
+
+// Optional phase timers (diagnostic builds only, -DLOSA_PHASE_TIMERS): clock64() deltas summed
+// per phase by one thread of each role and written to the workspace pointer at the end.
+#ifdef LOSA_PHASE_TIMERS
+#define PT_DECL() long long pt_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long pt_t = clock64()
+#define PT_MARK(i)                 \
+  do {                             \
+    const long long t_ = clock64(); \
+    pt_[i] += t_ - pt_t;           \
+    pt_t = t_;                     \
+  } while (0)
+#define PT_FLUSH(role)                                                                   \
+  do {                                                                                   \
+    if (MODE != kMass && p.table != nullptr && lane == 0) {                              \
+      long long* dst = reinterpret_cast<long long*>(p.table) + ((int64_t)blockIdx.x * 4 + (role)) * 8; \
+      for (int i_ = 0; i_ < 8; ++i_) dst[i_] = pt_[i_];                                  \
+    }                                                                                    \
+  } while (0)
+#else
+#define PT_DECL() do {} while (0)
+#define PT_MARK(i) do {} while (0)
+#define PT_FLUSH(role) do {} while (0)
+#endif
 
 #define LOSA_WAIT(bar, parity)                                   \
   do {                                                           \
@@ -205,18 +241,19 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       ptx::mbar_init(&ctl->q_full[i], 1);
       ptx::mbar_init(&ctl->q_empty[i], 1);
       ptx::mbar_init(&ctl->s_full[i], 1);
-      ptx::mbar_init(&ctl->p_ready[i], 128);
+      ptx::mbar_init(&ctl->p_ready[i][0], 4);  // one elected arrival per softmax warp
+      ptx::mbar_init(&ctl->p_ready[i][1], 4);
       ptx::mbar_init(&ctl->o_done[i], 1);
       ptx::mbar_init(&ctl->o_free[i], 128);
       ptx::mbar_init(&ctl->wg_bar[i], 128);
     }
     for (int i = 0; i < C::kNK; ++i) {
       ptx::mbar_init(&ctl->k_full[i], 1);
-      ptx::mbar_init(&ctl->k_empty[i], 1);
+      ptx::mbar_init(&ctl->k_empty[i], 2);  // both MMA issuers hand a stage back
     }
     for (int i = 0; i < C::kNV; ++i) {
       ptx::mbar_init(&ctl->v_full[i], 1);
-      ptx::mbar_init(&ctl->v_empty[i], 1);
+      ptx::mbar_init(&ctl->v_empty[i], 2);
     }
     ptx::mbar_init(&ctl->drain, 1);
     ctl->abort_flag = 0;
@@ -242,8 +279,10 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsUtility));
   if (warp == 8) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    // (the whole warp walks the tile list; lane 0 alone issues the copies)
+    {
       uint32_t nq[2] = {0, 0}, nk = 0, nv = 0;
+      PT_DECL();
       for (int w = blockIdx.x; w < p.nWork; w += gridDim.x) {
         const int bh = w / p.nPairs, pr = w % p.nPairs;
         const int b = bh / p.H, h = bh % p.H;
@@ -251,145 +290,169 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         for (int qt = 0; qt < 2; ++qt) {
           const int T = 2 * pr + qt;
           if (T < p.nQt) {
+            PT_MARK(0);
             LOSA_WAIT(&ctl->q_empty[qt], (nq[qt] & 1) ^ 1);
-            ptx::mbar_arrive_expect_tx(&ctl->q_full[qt], C::kQBytes);
+            PT_MARK(1);
+            if (lane == 0) {
+              ptx::mbar_arrive_expect_tx(&ctl->q_full[qt], C::kQBytes);
 #pragma unroll
-            for (int s = 0; s < C::kDH; ++s)
-              ptx::tma_load_4d(sQ + qt * C::kQBytes + s * C::kQSlab, &map_q, &ctl->q_full[qt],
-                               s * 64, T * 128, h, b);
+              for (int s = 0; s < C::kDH; ++s)
+                ptx::tma_load_4d(sQ + qt * C::kQBytes + s * C::kQSlab, &map_q, &ctl->q_full[qt],
+                                 s * 64, T * 128, h, b);
+            }
             ++nq[qt];
           }
         }
         TileIter<kNB> it;
-        it.init(p, MODE != kSparse, bh, 2 * pr * kQBT);
+        it.init(p, MODE != kSparse, bh, 2 * pr * kQBT, lane);
         int j;
         uint32_t memb;
         while (it.next(j, memb)) {
           const uint32_t ks = nk % C::kNK;
+          PT_MARK(0);
           LOSA_WAIT(&ctl->k_empty[ks], ((nk / C::kNK) & 1) ^ 1);
-          ptx::mbar_arrive_expect_tx(&ctl->k_full[ks], C::kKVBytes);
+          PT_MARK(2);
+          if (lane == 0) {
+            ptx::mbar_arrive_expect_tx(&ctl->k_full[ks], C::kKVBytes);
 #pragma unroll
-          for (int s = 0; s < C::kDH; ++s)
-            ptx::tma_load_4d(sK + ks * C::kKVBytes + s * C::kKVSlab, &map_k, &ctl->k_full[ks],
-                             s * 64, j * kC, h, b);
+            for (int s = 0; s < C::kDH; ++s)
+              ptx::tma_load_4d(sK + ks * C::kKVBytes + s * C::kKVSlab, &map_k, &ctl->k_full[ks],
+                               s * 64, j * kC, h, b);
+          }
           ++nk;
           if (C::kHasV) {
             const uint32_t vs = nv % (C::kNV > 0 ? C::kNV : 1);
+            PT_MARK(0);
             LOSA_WAIT(&ctl->v_empty[vs], ((nv / (C::kNV > 0 ? C::kNV : 1)) & 1) ^ 1);
-            ptx::mbar_arrive_expect_tx(&ctl->v_full[vs], C::kKVBytes);
+            PT_MARK(3);
+            if (lane == 0) {
+              ptx::mbar_arrive_expect_tx(&ctl->v_full[vs], C::kKVBytes);
 #pragma unroll
-            for (int s = 0; s < C::kDH; ++s)
-              ptx::tma_load_4d(sV + vs * C::kKVBytes + s * C::kKVSlab, &map_v, &ctl->v_full[vs],
-                               s * 64, j * kC, h, b);
+              for (int s = 0; s < C::kDH; ++s)
+                ptx::tma_load_4d(sV + vs * C::kKVBytes + s * C::kKVSlab, &map_v, &ctl->v_full[vs],
+                                 s * 64, j * kC, h, b);
+            }
             ++nv;
           }
         }
       }
+      PT_MARK(0);
+      PT_FLUSH(2);
     }
-  } else if (warp == 9) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+  } else if (warp == 9 || warp == 10) {
+    // ------------------------------------------------------------------ MMA issuers
+    // One issuing warp per query tile (warp 9: tile 0, warp 10: tile 1), so that a wait in one
+    // tile's chain never delays the other tile's MMAs.  Each walks every tile of the item in
+    // order (whole warp, for the shared index window); lane 0 alone issues MMAs and commits.
+    // For a tile its query tile does not list, the issuer only hands the K and V stages back.
+    {
+      const int qt = warp - 9;
+      const bool leader = (lane == 0);
       const uint32_t q_base = ptx::smem_u32(sQ), k_base = ptx::smem_u32(sK),
                      v_base = ptx::smem_u32(sV);
-      uint32_t nq[2] = {0, 0}, nk = 0, nv = 0, np[2] = {0, 0}, nof[2] = {0, 0};
+      uint32_t nq = 0, nt = 0, np = 0, nof = 0;  // nt: tiles walked since the kernel started
+      PT_DECL();
 
-      auto issue_qk = [&](int qt, uint32_t ks) {
-        const uint32_t a0 = q_base + qt * C::kQBytes, b0 = k_base + ks * C::kKVBytes;
+      // Descriptor low words of every buffer, computed once; per MMA only a constant is added.
+      constexpr uint32_t kDescHi = ptx::smem_desc_hi_sw128(1024);
+      const uint32_t q_lo = ptx::smem_desc_lo(q_base, 16) + qt * (C::kQBytes >> 4);
+      const uint32_t k_lo = ptx::smem_desc_lo(k_base, 16);
+      const uint32_t v_lo = ptx::smem_desc_lo(v_base, C::kKVSlab);
+      const uint32_t tS = tmem_base + qt * 128, tO = tmem_base + 256 + qt * 128;
+      auto issue_qk = [&](uint32_t ks) {
+        if (!leader) return;
+        const uint32_t b0 = k_lo + ks * (C::kKVBytes >> 4);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk & 3) * 32;
-          const uint64_t ad = ptx::smem_desc_sw128(a0 + (kk >> 2) * C::kQSlab + off, 16, 1024);
-          const uint64_t bd = ptx::smem_desc_sw128(b0 + (kk >> 2) * C::kKVSlab + off, 16, 1024);
-          ptx::mma_ss(tmem_base + qt * 128, ad, bd, C::kIdescQK, kk > 0 ? 1u : 0u);
+          const uint32_t a_off = ((kk >> 2) * C::kQSlab + (kk & 3) * 32) >> 4;
+          const uint32_t b_off = ((kk >> 2) * C::kKVSlab + (kk & 3) * 32) >> 4;
+          ptx::mma_ss_lohi(tS, q_lo + a_off, b0 + b_off, kDescHi, C::kIdescQK, kk > 0 ? 1u : 0u);
         }
       };
-      auto issue_pv = [&](int qt, uint32_t vs, bool accumulate) {
-        const uint32_t b0 = v_base + vs * C::kKVBytes;
+      auto issue_pv = [&](uint32_t vs, bool accumulate, int half) {
+        if (!leader) return;
+        const uint32_t b0 = v_lo + vs * (C::kKVBytes >> 4);
 #pragma unroll
-        for (int kk = 0; kk < kC / 16; ++kk) {
-          const uint64_t bd = ptx::smem_desc_sw128(b0 + kk * 2048, C::kKVSlab, 1024);
-          ptx::mma_ts(tmem_base + 256 + qt * 128, tmem_base + qt * 128 + kk * 8, bd, C::kIdescPV,
-                      (accumulate || kk > 0) ? 1u : 0u);
+        for (int k2 = 0; k2 < kC / 32; ++k2) {
+          const int kk = half * (kC / 32) + k2;
+          ptx::mma_ts_lohi(tO, tS + kk * 8, b0 + kk * (2048 >> 4), kDescHi, C::kIdescPV,
+                           (accumulate || k2 > 0) ? 1u : 0u);
         }
       };
+      constexpr uint32_t kNVs = C::kNV > 0 ? C::kNV : 1;
 
       for (int w = blockIdx.x; w < p.nWork; w += gridDim.x) {
         const int bh = w / p.nPairs, pr = w % p.nPairs;
         TileIter<kNB> it;
-        it.init(p, MODE != kSparse, bh, 2 * pr * kQBT);
-        bool q_ready[2] = {false, false};
-        uint32_t pv_item[2] = {0, 0};
-        int jc;
-        uint32_t mc;
-        bool have = it.next(jc, mc);
-        if (have) {
-          const uint32_t ks = nk % C::kNK;
-          LOSA_WAIT(&ctl->k_full[ks], (nk / C::kNK) & 1);
-#pragma unroll
-          for (int qt = 0; qt < 2; ++qt) {
-            if ((mc >> (qt * kQBT)) & kQMask) {
-              LOSA_WAIT(&ctl->q_full[qt], nq[qt] & 1);
-              ++nq[qt];
-              q_ready[qt] = true;
-              ptx::tc_fence_after_sync();
-              issue_qk(qt, ks);
-              ptx::mma_commit(&ctl->s_full[qt]);
-            }
-          }
-          ptx::mma_commit(&ctl->k_empty[ks]);
-          ++nk;
-        }
+        it.init(p, MODE != kSparse, bh, 2 * pr * kQBT, lane);
+        bool q_ready = false;
+        uint32_t pv_item = 0;
+        int j;
+        uint32_t memb;
+        bool have = it.next(j, memb);
         while (have) {
-          int jn;
-          uint32_t mn;
-          const bool have_n = it.next(jn, mn);
-          const uint32_t ksn = nk % C::kNK;
-          const uint32_t vs = nv % (C::kNV > 0 ? C::kNV : 1);
-          if (have_n) LOSA_WAIT(&ctl->k_full[ksn], (nk / C::kNK) & 1);
-          if (C::kHasV) LOSA_WAIT(&ctl->v_full[vs], (nv / (C::kNV > 0 ? C::kNV : 1)) & 1);
-#pragma unroll
-          for (int qt = 0; qt < 2; ++qt) {
-            if ((mc >> (qt * kQBT)) & kQMask) {
-              LOSA_WAIT(&ctl->p_ready[qt], np[qt] & 1);
-              ++np[qt];
-              if (C::kHasV) {
-                if (pv_item[qt] == 0 && nof[qt] > 0)
-                  LOSA_WAIT(&ctl->o_free[qt], (nof[qt] - 1) & 1);
-                ptx::tc_fence_after_sync();
-                issue_pv(qt, vs, pv_item[qt] > 0);
-                ptx::mma_commit(&ctl->o_done[qt]);
-                ++pv_item[qt];
-              }
+          const uint32_t ks = nt % C::kNK, kph = (nt / C::kNK) & 1;
+          const uint32_t vs = nt % kNVs, vph = (nt / kNVs) & 1;
+          const bool member = ((memb >> (qt * kQBT)) & kQMask) != 0;
+          PT_MARK(0);
+          LOSA_WAIT(&ctl->k_full[ks], kph);
+          PT_MARK(1);
+          if (member) {
+            if (!q_ready) {
+              LOSA_WAIT(&ctl->q_full[qt], nq & 1);
+              ++nq;
+              q_ready = true;
             }
-            if (have_n && ((mn >> (qt * kQBT)) & kQMask)) {
-              if (!q_ready[qt]) {
-                LOSA_WAIT(&ctl->q_full[qt], nq[qt] & 1);
-                ++nq[qt];
-                q_ready[qt] = true;
-              }
-              ptx::tc_fence_after_sync();
-              issue_qk(qt, ksn);
+            ptx::tc_fence_after_sync();
+            issue_qk(ks);
+            PT_MARK(5);
+            if (leader) {
               ptx::mma_commit(&ctl->s_full[qt]);
+              ptx::mma_commit(&ctl->k_empty[ks]);
             }
+            PT_MARK(6);
+          } else if (leader) {
+            ptx::mbar_arrive(&ctl->k_empty[ks]);
           }
+          // walk ahead while the softmax warpgroup works on this tile
+          have = it.next(j, memb);
+          PT_MARK(0);
           if (C::kHasV) {
-            ptx::mma_commit(&ctl->v_empty[vs]);
-            ++nv;
+            LOSA_WAIT(&ctl->v_full[vs], vph);
+            PT_MARK(1);
           }
-          if (have_n) {
-            ptx::mma_commit(&ctl->k_empty[ksn]);
-            ++nk;
+          if (member) {
+            LOSA_WAIT(&ctl->p_ready[qt][0], np & 1);
+            PT_MARK(2);
+            if (C::kHasV) {
+              if (pv_item == 0 && nof > 0) LOSA_WAIT(&ctl->o_free[qt], (nof - 1) & 1);
+              ptx::tc_fence_after_sync();
+              issue_pv(vs, pv_item > 0, 0);  // keys of the first half of P
+              PT_MARK(4);
+              LOSA_WAIT(&ctl->p_ready[qt][1], np & 1);
+              PT_MARK(2);
+              ptx::tc_fence_after_sync();
+              issue_pv(vs, true, 1);
+              PT_MARK(4);
+              ++pv_item;
+            }
+            ++np;
           }
-          have = have_n;
-          mc = mn;
-          jc = jn;
+          if (C::kHasV && leader) {
+            if (member) ptx::mma_commit(&ctl->v_empty[vs]);
+            else ptx::mbar_arrive(&ctl->v_empty[vs]);
+          }
+          PT_MARK(6);
+          ++nt;
         }
-#pragma unroll
-        for (int qt = 0; qt < 2; ++qt) {
-          if (q_ready[qt]) ptx::mma_commit(&ctl->q_empty[qt]);
-          if (pv_item[qt] > 0) ++nof[qt];
+        if (q_ready && leader) ptx::mma_commit(&ctl->q_empty[qt]);
+        if (pv_item > 0) {
+          if (leader) ptx::mma_commit(&ctl->o_done[qt]);  // every PV of the item is done
+          ++nof;
         }
       }
+      PT_MARK(0);
+      if (qt == 0) PT_FLUSH(3);
     }
   }
   } else {
@@ -403,7 +466,8 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int sub = (BLK == 64) ? (wl >> 1) : 0;
     const int my_bit = qt * kQBT + sub;
     const int tail = p.N - (p.nKb - 1) * kC;  // valid keys of the last K/V tile
-    uint32_t ns = 0, npv = 0, nwg = 0;
+    uint32_t ns = 0, npv = 0, nwg = 0;  // npv: items of this query tile whose O was read out
+    PT_DECL();
 
     for (int w = blockIdx.x; w < p.nWork; w += gridDim.x) {
       const int bh = w / p.nPairs, pr = w % p.nPairs;
@@ -411,7 +475,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const int T = 2 * pr + qt;
       const int grow = T * 128 + row;
       TileIter<kNB> it;
-      it.init(p, MODE != kSparse, bh, 2 * pr * kQBT);
+      it.init(p, MODE != kSparse, bh, 2 * pr * kQBT, lane);
       float m_ref = -INFINITY, l = 0.f;
       uint32_t pv_item = 0;
       float2* tab = nullptr;
@@ -421,7 +485,9 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       uint32_t memb;
       while (it.next(j, memb)) {
         if (((memb >> (qt * kQBT)) & kQMask) == 0) continue;
+        PT_MARK(0);
         LOSA_WAIT(&ctl->s_full[qt], ns & 1);
+        PT_MARK(1);
         ++ns;
         ptx::tc_fence_after_sync();
         const bool mine = (memb >> my_bit) & 1u;
@@ -430,6 +496,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
           for (int c0 = 0; c0 < kC; c0 += 32) ptx::tmem_ld32(tS + c0, &sr[c0]);
           ptx::tmem_wait_ld();
+          PT_MARK(2);
           if (j == p.nKb - 1 && tail < kC) {
 #pragma unroll
             for (int c = 0; c < kC; ++c)
@@ -438,12 +505,14 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
           float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
 #pragma unroll
-          for (int c = 4; c < kC; c += 4) {
-            mx0 = fmaxf(mx0, __uint_as_float(sr[c]));
-            mx1 = fmaxf(mx1, __uint_as_float(sr[c + 1]));
-            mx2 = fmaxf(mx2, __uint_as_float(sr[c + 2]));
-            mx3 = fmaxf(mx3, __uint_as_float(sr[c + 3]));
+          for (int c = 4; c + 8 <= kC; c += 8) {
+            mx0 = ptx::max3(mx0, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
+            mx1 = ptx::max3(mx1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
+            mx2 = ptx::max3(mx2, __uint_as_float(sr[c + 4]), __uint_as_float(sr[c + 5]));
+            mx3 = ptx::max3(mx3, __uint_as_float(sr[c + 6]), __uint_as_float(sr[c + 7]));
           }
+          mx0 = ptx::max3(mx0, __uint_as_float(sr[kC - 4]), __uint_as_float(sr[kC - 3]));
+          mx1 = ptx::max3(mx1, __uint_as_float(sr[kC - 2]), __uint_as_float(sr[kC - 1]));
           const float m_new = fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
           const bool need = m_new > m_ref + kRescaleThreshold;
           if (__any_sync(0xffffffffu, need)) {
@@ -451,8 +520,8 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             if (need) m_ref = m_new;
             l *= alpha;
             if (C::kHasV && pv_item > 0) {
-              LOSA_WAIT(&ctl->o_done[qt], (npv - 1) & 1);
-              ptx::tc_fence_after_sync();
+              // O is stable here: S of this tile was committed after the previous PV of this
+              // query tile in the same in-order MMA stream, so that PV has completed.
               const float2 a2 = make_float2(alpha, alpha);
 #pragma unroll
               for (int c0 = 0; c0 < D; c0 += 32) {
@@ -472,44 +541,71 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
           // p = 2^(s * scale_log2 - m_ref), two columns per instruction; the bf16 pair replaces
           // the first of the two fp32 registers
+          PT_MARK(3);
           const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
           const float2 nm2 = make_float2(-m_ref, -m_ref);
           float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+          // two halves of the key tile: the first half of P is handed to the MMA thread while
+          // the second half is still being exponentiated
 #pragma unroll
-          for (int c = 0; c < kC; c += 4) {
-            float2 x0 = ptx::fma2(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2);
-            float2 x1 = ptx::fma2(make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, nm2);
-            x0.x = ptx::ex2_approx(x0.x);
-            x0.y = ptx::ex2_approx(x0.y);
-            x1.x = ptx::ex2_approx(x1.x);
-            x1.y = ptx::ex2_approx(x1.y);
-            acc0 = ptx::add2(acc0, x0);
-            acc1 = ptx::add2(acc1, x1);
-            sr[c >> 1] = ptx::pack_bf16x2(x0.x, x0.y);
-            sr[(c >> 1) + 1] = ptx::pack_bf16x2(x1.x, x1.y);
+          for (int half = 0; half < 2; ++half) {
+#pragma unroll
+            for (int c = half * (kC / 2); c < (half + 1) * (kC / 2); c += 4) {
+              float2 x0 = ptx::fma2(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2);
+              float2 x1 = ptx::fma2(make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, nm2);
+              x0.x = ptx::ex2_approx(x0.x);
+              x0.y = ptx::ex2_approx(x0.y);
+              x1.x = ptx::ex2_approx(x1.x);
+              x1.y = ptx::ex2_approx(x1.y);
+              acc0 = ptx::add2(acc0, x0);
+              acc1 = ptx::add2(acc1, x1);
+              sr[c >> 1] = ptx::pack_bf16x2(x0.x, x0.y);
+              sr[(c >> 1) + 1] = ptx::pack_bf16x2(x1.x, x1.y);
+            }
+            if (C::kHasV) {
+              if (kC == 128) ptx::tmem_st32(tS + half * 32, &sr[half * 32]);
+              else ptx::tmem_st16(tS + half * 16, &sr[half * 16]);
+#ifdef LOSA_X_LATE_P0
+              if (half == 1) {
+#else
+              if (half == 0) {
+#endif
+                ptx::tmem_wait_st();
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&ctl->p_ready[qt][0]);
+              }
+            }
           }
+          PT_MARK(4);
           const float tsum = (acc0.x + acc0.y) + (acc1.x + acc1.y);
           l += tsum;
-          if (C::kHasV) {
-#pragma unroll
-            for (int c0 = 0; c0 < kC / 2; c0 += 32) ptx::tmem_st32(tS + c0, &sr[c0]);
-          } else {
-            tab[(int64_t)j * 128] = make_float2(tsum, m_ref);
-          }
+          if (!C::kHasV) tab[(int64_t)j * 128] = make_float2(tsum, m_ref);
         } else if (C::kHasV) {
+          // this half of the 128-row tile does not list the key block: P = 0
           uint32_t z[32];
 #pragma unroll
           for (int c = 0; c < 32; ++c) z[c] = 0u;
-#pragma unroll
-          for (int c0 = 0; c0 < kC / 2; c0 += 32) ptx::tmem_st32(tS + c0, z);
+          if (kC == 128) {
+            ptx::tmem_st32(tS, z);
+            ptx::tmem_st32(tS + 32, z);
+          } else {
+            ptx::tmem_st32(tS, z);
+          }
+          ptx::tmem_wait_st();
+          ptx::tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&ctl->p_ready[qt][0]);
         }
         if (C::kHasV) {
           ptx::tmem_wait_st();
           ++pv_item;
-          ++npv;
         }
         ptx::tc_fence_before_sync();
-        ptx::mbar_arrive(&ctl->p_ready[qt]);
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&ctl->p_ready[qt][C::kHasV ? 1 : 0]);
+
+        PT_MARK(5);
       }
 
       if (MODE != kMass) {
@@ -519,7 +615,8 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const float inv = (l > 0.f) ? 1.f / l : 0.f;
           const int64_t off = (int64_t)b * p.sb + (int64_t)h * p.sh + (int64_t)grow * p.sn;
           if (pv_item > 0) {
-            LOSA_WAIT(&ctl->o_done[qt], (npv - 1) & 1);
+            LOSA_WAIT(&ctl->o_done[qt], npv & 1);
+            ++npv;
             ptx::tc_fence_after_sync();
           }
 #pragma unroll
@@ -602,14 +699,16 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         LOSA_WAIT(&ctl->wg_bar[qt], nwg & 1);
         ++nwg;
       }
+      PT_MARK(6);  // epilogue of the item
     }
+    if (wl == 0) PT_FLUSH(qt);
   }
 
 teardown:
   if (ctl->abort_flag) {
     // Abort path: give MMAs and bulk copies still in flight a bounded time to land before
     // shared memory and TMEM are released.
-    if (warp == 9 && lane == 0) {
+    if ((warp == 9 || warp == 10) && lane == 0) {
       ptx::mma_commit(&ctl->drain);
       for (uint32_t it = 0; it < (1u << 16); ++it) {
         if (ptx::mbar_try_wait(&ctl->drain, 0)) break;
