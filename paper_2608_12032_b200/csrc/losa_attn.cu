@@ -62,12 +62,13 @@ struct Cfg {
   static constexpr int kNV = kHasV ? ((kKVBytes >= 32768) ? 2 : 4) : 0;
   static constexpr int kNK0 = (kRingBudget - kNV * kKVBytes) / kKVBytes;
   static constexpr int kNK = kNK0 > 6 ? 6 : kNK0;
-  static constexpr uint32_t kIdescQK = ptx::idesc_bf16_f32(128, kC, false, false);
+  static constexpr uint32_t kIdescQK = ptx::idesc_bf16_f32(128, 64, false, false);  // 64-key sub-tile
   static constexpr uint32_t kIdescPV = ptx::idesc_bf16_f32(128, D, false, true);
 };
 
 struct Params {
   int B, H, N, nQb, nKb, nQt, nPairs, nWork;
+  int tail_subs;  // 64-key sub-tiles of the last key tile that hold valid keys
   const int32_t* offsets;
   const int32_t* kv_idx;
   void* o;
@@ -75,7 +76,7 @@ struct Params {
   int64_t sb, sh, sn;
   float* mass;
   float* lse;
-  float2* table;  // mass mode: [grid][2][nKb][128] (sum of p, reference max) per row and tile
+  float2* table;  // mass mode: [grid][2][nKb * C/64][128] (sum of p, reference max) per row and sub-tile
   float scale_log2;
   int* status;
 };
@@ -85,7 +86,8 @@ struct Control {
   uint64_t q_full[2], q_empty[2];
   uint64_t k_full[NK], k_empty[NK];
   uint64_t v_full[NV > 0 ? NV : 1], v_empty[NV > 0 ? NV : 1];
-  uint64_t s_full[2], p_ready[2][2], o_done[2], o_free[2];  // p_ready: one per half of P
+  uint64_t s_full[2][2], p_ready[2][2];  // per query tile and S buffer
+  uint64_t pv_done[2], o_done[2], o_free[2];  // per product / per item / O read out
   uint64_t wg_bar[2];
   uint64_t drain;
   uint32_t tmem_base;
@@ -240,9 +242,11 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(&ctl->q_full[i], 1);
       ptx::mbar_init(&ctl->q_empty[i], 1);
-      ptx::mbar_init(&ctl->s_full[i], 1);
+      ptx::mbar_init(&ctl->s_full[i][0], 1);
+      ptx::mbar_init(&ctl->s_full[i][1], 1);
       ptx::mbar_init(&ctl->p_ready[i][0], 4);  // one elected arrival per softmax warp
       ptx::mbar_init(&ctl->p_ready[i][1], 4);
+      ptx::mbar_init(&ctl->pv_done[i], 1);
       ptx::mbar_init(&ctl->o_done[i], 1);
       ptx::mbar_init(&ctl->o_free[i], 128);
       ptx::mbar_init(&ctl->wg_bar[i], 128);
@@ -344,113 +348,141 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // One issuing warp per query tile (warp 9: tile 0, warp 10: tile 1), so that a wait in one
     // tile's chain never delays the other tile's MMAs.  Each walks every tile of the item in
     // order (whole warp, for the shared index window); lane 0 alone issues MMAs and commits.
-    // For a tile its query tile does not list, the issuer only hands the K and V stages back.
+    //
+    // A key tile is consumed as 64-key sub-tiles, and the S accumulator of a query tile is
+    // double-buffered (2 x 64 TMEM columns): S(n+1) = Q K(n+1)^T is issued before O += P(n) V(n),
+    // so the tensor pipe works on sub-tile n+1 and n-1 while the softmax warpgroup is busy
+    // with sub-tile n.  Up to two P V products are pending at any time.
     {
       const int qt = warp - 9;
       const bool leader = (lane == 0);
       const uint32_t q_base = ptx::smem_u32(sQ), k_base = ptx::smem_u32(sK),
                      v_base = ptx::smem_u32(sV);
-      uint32_t nq = 0, nt = 0, np = 0, nof = 0;  // nt: tiles walked since the kernel started
+      uint32_t nq = 0, nt = 0, nsub = 0, npv = 0, nof = 0;
+      // nt: tiles walked, nsub: S sub-tiles issued, npv: P V products issued (kernel lifetime)
       PT_DECL();
 
-      // Descriptor low words of every buffer, computed once; per MMA only a constant is added.
       constexpr uint32_t kDescHi = ptx::smem_desc_hi_sw128(1024);
       const uint32_t q_lo = ptx::smem_desc_lo(q_base, 16) + qt * (C::kQBytes >> 4);
       const uint32_t k_lo = ptx::smem_desc_lo(k_base, 16);
       const uint32_t v_lo = ptx::smem_desc_lo(v_base, C::kKVSlab);
       const uint32_t tS = tmem_base + qt * 128, tO = tmem_base + 256 + qt * 128;
-      auto issue_qk = [&](uint32_t ks) {
+      constexpr uint32_t kNVs = C::kNV > 0 ? C::kNV : 1;
+
+      // S[buf] = Q K(stage ks, keys 64 h .. 64 h + 63)^T
+      auto issue_qk = [&](uint32_t ks, int h, uint32_t buf) {
         if (!leader) return;
-        const uint32_t b0 = k_lo + ks * (C::kKVBytes >> 4);
+        const uint32_t b0 = k_lo + ks * (C::kKVBytes >> 4) + ((h * 64 * 128) >> 4);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t a_off = ((kk >> 2) * C::kQSlab + (kk & 3) * 32) >> 4;
           const uint32_t b_off = ((kk >> 2) * C::kKVSlab + (kk & 3) * 32) >> 4;
-          ptx::mma_ss_lohi(tS, q_lo + a_off, b0 + b_off, kDescHi, C::kIdescQK, kk > 0 ? 1u : 0u);
+          ptx::mma_ss_lohi(tS + buf * 64, q_lo + a_off, b0 + b_off, kDescHi, C::kIdescQK,
+                           kk > 0 ? 1u : 0u);
         }
       };
-      auto issue_pv = [&](uint32_t vs, bool accumulate, int half) {
+      // O (+)= P[buf] V(stage vs, keys 64 h .. 64 h + 63)
+      auto issue_pv = [&](uint32_t vs, int h, uint32_t buf, bool accumulate) {
         if (!leader) return;
-        const uint32_t b0 = v_lo + vs * (C::kKVBytes >> 4);
+        const uint32_t b0 = v_lo + vs * (C::kKVBytes >> 4) + ((h * 64 * 128) >> 4);
 #pragma unroll
-        for (int k2 = 0; k2 < kC / 32; ++k2) {
-          const int kk = half * (kC / 32) + k2;
-          ptx::mma_ts_lohi(tO, tS + kk * 8, b0 + kk * (2048 >> 4), kDescHi, C::kIdescPV,
-                           (accumulate || k2 > 0) ? 1u : 0u);
-        }
+        for (int kk = 0; kk < 4; ++kk)
+          ptx::mma_ts_lohi(tO, tS + buf * 64 + kk * 8, b0 + kk * (2048 >> 4), kDescHi,
+                           C::kIdescPV, (accumulate || kk > 0) ? 1u : 0u);
       };
-      constexpr uint32_t kNVs = C::kNV > 0 ? C::kNV : 1;
+
+      // pending P V products, oldest first: V stage, its phase, sub-tile, last-of-tile flag
+      // (kept in scalars: slot 0 is the oldest, slot 1 the newest)
+      uint32_t pd_vs0 = 0, pd_ph0 = 0, pd_tile0 = 0, pd_vs1 = 0, pd_ph1 = 0, pd_tile1 = 0;
+      int pd_h0 = 0, pd_h1 = 0;
+      bool pd_last0 = false, pd_last1 = false;
+      int npend = 0;
+      uint32_t pv_item = 0;
+
+#define LOSA_POP_PV()                                                              \
+  do {                                                                             \
+    PT_MARK(0);                                                                    \
+    if (C::kHasV) LOSA_WAIT(&ctl->v_full[pd_vs0], pd_ph0);                     \
+    PT_MARK(1);                                                                    \
+    LOSA_WAIT(&ctl->p_ready[qt][npv & 1], (npv >> 1) & 1);                         \
+    PT_MARK(2);                                                                    \
+    if (C::kHasV) {                                                                \
+      if (pv_item == 0 && nof > 0) LOSA_WAIT(&ctl->o_free[qt], (nof - 1) & 1);     \
+      ptx::tc_fence_after_sync();                                                  \
+      issue_pv(pd_vs0, pd_h0, npv & 1, pv_item > 0);                           \
+      PT_MARK(4);                                                                  \
+      if (leader) {                                                                \
+        ptx::mma_commit(&ctl->pv_done[qt]);                                        \
+        if (pd_last0) ptx::mma_commit(&ctl->v_empty[pd_vs0]);                  \
+      }                                                                            \
+      ++pv_item;                                                                   \
+    }                                                                              \
+    ++npv;                                                                         \
+    pd_vs0 = pd_vs1; pd_ph0 = pd_ph1; pd_h0 = pd_h1;                               \
+    pd_last0 = pd_last1; pd_tile0 = pd_tile1;                                      \
+    --npend;                                                                       \
+    PT_MARK(6);                                                                    \
+  } while (0)
 
       for (int w = blockIdx.x; w < p.nWork; w += gridDim.x) {
         const int bh = w / p.nPairs, pr = w % p.nPairs;
         TileIter<kNB> it;
         it.init(p, MODE != kSparse, bh, 2 * pr * kQBT, lane);
         bool q_ready = false;
-        uint32_t pv_item = 0;
+        pv_item = 0;
         int j;
         uint32_t memb;
-        bool have = it.next(j, memb);
-        while (have) {
+        while (it.next(j, memb)) {
           const uint32_t ks = nt % C::kNK, kph = (nt / C::kNK) & 1;
           const uint32_t vs = nt % kNVs, vph = (nt / kNVs) & 1;
           const bool member = ((memb >> (qt * kQBT)) & kQMask) != 0;
+          const int subs = (j == p.nKb - 1) ? p.tail_subs : (kC / 64);
           PT_MARK(0);
           LOSA_WAIT(&ctl->k_full[ks], kph);
           PT_MARK(1);
+          // V stages go back to the producer in tile order, and the producer refills this
+          // tile's stage only after its previous user was handed back: finish the pending
+          // products of any tile that used this V stage before.
+          while (C::kHasV && npend > 0 && pd_tile0 + kNVs <= nt) LOSA_POP_PV();
           if (member) {
             if (!q_ready) {
               LOSA_WAIT(&ctl->q_full[qt], nq & 1);
               ++nq;
               q_ready = true;
             }
-            ptx::tc_fence_after_sync();
-            issue_qk(ks);
-            PT_MARK(5);
-            if (leader) {
-              ptx::mma_commit(&ctl->s_full[qt]);
-              ptx::mma_commit(&ctl->k_empty[ks]);
+            for (int h = 0; h < subs; ++h) {
+              if (npend == 2) LOSA_POP_PV();  // frees the S buffer this sub-tile will use
+              ptx::tc_fence_after_sync();
+              issue_qk(ks, h, nsub & 1);
+              PT_MARK(5);
+              if (leader) ptx::mma_commit(&ctl->s_full[qt][nsub & 1]);
+              if (npend == 0) {
+                pd_vs0 = vs; pd_ph0 = vph; pd_h0 = h; pd_tile0 = nt; pd_last0 = (h == subs - 1);
+              } else {
+                pd_vs1 = vs; pd_ph1 = vph; pd_h1 = h; pd_tile1 = nt; pd_last1 = (h == subs - 1);
+              }
+              ++npend;
+              ++nsub;
+              PT_MARK(6);
             }
-            PT_MARK(6);
-          } else if (leader) {
-            ptx::mbar_arrive(&ctl->k_empty[ks]);
-          }
-          // walk ahead while the softmax warpgroup works on this tile
-          have = it.next(j, memb);
-          PT_MARK(0);
-          if (C::kHasV) {
-            LOSA_WAIT(&ctl->v_full[vs], vph);
-            PT_MARK(1);
-          }
-          if (member) {
-            LOSA_WAIT(&ctl->p_ready[qt][0], np & 1);
-            PT_MARK(2);
+            if (leader) ptx::mma_commit(&ctl->k_empty[ks]);
+          } else {
+            if (leader) ptx::mbar_arrive(&ctl->k_empty[ks]);
             if (C::kHasV) {
-              if (pv_item == 0 && nof > 0) LOSA_WAIT(&ctl->o_free[qt], (nof - 1) & 1);
-              ptx::tc_fence_after_sync();
-              issue_pv(vs, pv_item > 0, 0);  // keys of the first half of P
-              PT_MARK(4);
-              LOSA_WAIT(&ctl->p_ready[qt][1], np & 1);
-              PT_MARK(2);
-              ptx::tc_fence_after_sync();
-              issue_pv(vs, true, 1);
-              PT_MARK(4);
-              ++pv_item;
+              LOSA_WAIT(&ctl->v_full[vs], vph);
+              if (leader) ptx::mbar_arrive(&ctl->v_empty[vs]);
             }
-            ++np;
           }
-          if (C::kHasV && leader) {
-            if (member) ptx::mma_commit(&ctl->v_empty[vs]);
-            else ptx::mbar_arrive(&ctl->v_empty[vs]);
-          }
-          PT_MARK(6);
           ++nt;
         }
+        while (npend > 0) LOSA_POP_PV();
         if (q_ready && leader) ptx::mma_commit(&ctl->q_empty[qt]);
         if (pv_item > 0) {
-          if (leader) ptx::mma_commit(&ctl->o_done[qt]);  // every PV of the item is done
+          if (leader) ptx::mma_commit(&ctl->o_done[qt]);  // every product of the item is done
           ++nof;
         }
       }
+#undef LOSA_POP_PV
       PT_MARK(0);
       if (qt == 0) PT_FLUSH(3);
     }
@@ -466,7 +498,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int sub = (BLK == 64) ? (wl >> 1) : 0;
     const int my_bit = qt * kQBT + sub;
     const int tail = p.N - (p.nKb - 1) * kC;  // valid keys of the last K/V tile
-    uint32_t ns = 0, npv = 0, nwg = 0;  // npv: items of this query tile whose O was read out
+    uint32_t nsub = 0, nwg = 0, nod = 0;      // nsub: sub-tiles of this query tile so far
     PT_DECL();
 
     for (int w = blockIdx.x; w < p.nWork; w += gridDim.x) {
@@ -480,79 +512,85 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       uint32_t pv_item = 0;
       float2* tab = nullptr;
       if (MODE == kMass)
-        tab = p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * 128 + row;
+        tab = p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * (kC / 64) * 128 + row;
       int j;
       uint32_t memb;
       while (it.next(j, memb)) {
         if (((memb >> (qt * kQBT)) & kQMask) == 0) continue;
-        PT_MARK(0);
-        LOSA_WAIT(&ctl->s_full[qt], ns & 1);
-        PT_MARK(1);
-        ++ns;
-        ptx::tc_fence_after_sync();
         const bool mine = (memb >> my_bit) & 1u;
-        if (mine) {
-          uint32_t sr[kC];
+        const int subs = (j == p.nKb - 1) ? p.tail_subs : (kC / 64);
+        for (int hs = 0; hs < subs; ++hs) {
+          const uint32_t buf = nsub & 1, ph = (nsub >> 1) & 1;
+          const uint32_t tSb = tS + buf * 64;
+          PT_MARK(0);
+          LOSA_WAIT(&ctl->s_full[qt][buf], ph);
+          PT_MARK(1);
+          ptx::tc_fence_after_sync();
+          if (mine) {
+            uint32_t sr[64];
+            ptx::tmem_ld32(tSb, &sr[0]);
+            ptx::tmem_ld32(tSb + 32, &sr[32]);
+            ptx::tmem_wait_ld();
+            PT_MARK(2);
+            if (j == p.nKb - 1) {
+              const int valid = tail - hs * 64;  // keys >= N do not exist
+              if (valid < 64) {
 #pragma unroll
-          for (int c0 = 0; c0 < kC; c0 += 32) ptx::tmem_ld32(tS + c0, &sr[c0]);
-          ptx::tmem_wait_ld();
-          PT_MARK(2);
-          if (j == p.nKb - 1 && tail < kC) {
-#pragma unroll
-            for (int c = 0; c < kC; ++c)
-              if (c >= tail) sr[c] = 0xff800000u;  // -inf: the key does not exist
-          }
-          float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
-          float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
-#pragma unroll
-          for (int c = 4; c + 8 <= kC; c += 8) {
-            mx0 = ptx::max3(mx0, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
-            mx1 = ptx::max3(mx1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
-            mx2 = ptx::max3(mx2, __uint_as_float(sr[c + 4]), __uint_as_float(sr[c + 5]));
-            mx3 = ptx::max3(mx3, __uint_as_float(sr[c + 6]), __uint_as_float(sr[c + 7]));
-          }
-          mx0 = ptx::max3(mx0, __uint_as_float(sr[kC - 4]), __uint_as_float(sr[kC - 3]));
-          mx1 = ptx::max3(mx1, __uint_as_float(sr[kC - 2]), __uint_as_float(sr[kC - 1]));
-          const float m_new = fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
-          const bool need = m_new > m_ref + kRescaleThreshold;
-          if (__any_sync(0xffffffffu, need)) {
-            const float alpha = need ? ptx::ex2_approx(m_ref - m_new) : 1.f;
-            if (need) m_ref = m_new;
-            l *= alpha;
-            if (C::kHasV && pv_item > 0) {
-              // O is stable here: S of this tile was committed after the previous PV of this
-              // query tile in the same in-order MMA stream, so that PV has completed.
-              const float2 a2 = make_float2(alpha, alpha);
-#pragma unroll
-              for (int c0 = 0; c0 < D; c0 += 32) {
-                uint32_t r[32];
-                ptx::tmem_ld32(tO + c0, r);
-                ptx::tmem_wait_ld();
-#pragma unroll
-                for (int c = 0; c < 32; c += 2) {
-                  const float2 v = ptx::mul2(
-                      make_float2(__uint_as_float(r[c]), __uint_as_float(r[c + 1])), a2);
-                  r[c] = __float_as_uint(v.x);
-                  r[c + 1] = __float_as_uint(v.y);
-                }
-                ptx::tmem_st32(tO + c0, r);
+                for (int c = 0; c < 64; ++c)
+                  if (c >= valid) sr[c] = 0xff800000u;
               }
             }
-          }
-          // p = 2^(s * scale_log2 - m_ref), two columns per instruction; the bf16 pair replaces
-          // the first of the two fp32 registers
-          PT_MARK(3);
-          const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
-          const float2 nm2 = make_float2(-m_ref, -m_ref);
-          float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-          // two halves of the key tile: the first half of P is handed to the MMA thread while
-          // the second half is still being exponentiated
+            float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
+            float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
+            for (int c = 4; c + 8 <= 64; c += 8) {
+              mx0 = ptx::max3(mx0, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
+              mx1 = ptx::max3(mx1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
+              mx2 = ptx::max3(mx2, __uint_as_float(sr[c + 4]), __uint_as_float(sr[c + 5]));
+              mx3 = ptx::max3(mx3, __uint_as_float(sr[c + 6]), __uint_as_float(sr[c + 7]));
+            }
+            mx0 = ptx::max3(mx0, __uint_as_float(sr[60]), __uint_as_float(sr[61]));
+            mx1 = ptx::max3(mx1, __uint_as_float(sr[62]), __uint_as_float(sr[63]));
+            const float m_new =
+                fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
+            const bool need = m_new > m_ref + kRescaleThreshold;
+            if (__any_sync(0xffffffffu, need)) {
+              const float alpha = need ? ptx::ex2_approx(m_ref - m_new) : 1.f;
+              if (need) m_ref = m_new;
+              l *= alpha;
+              if (C::kHasV && pv_item > 0) {
+                // O may only be touched once the previous product of this query tile is done
+                LOSA_WAIT(&ctl->pv_done[qt], (nsub - 1) & 1);
+                ptx::tc_fence_after_sync();
+                const float2 a2 = make_float2(alpha, alpha);
 #pragma unroll
-            for (int c = half * (kC / 2); c < (half + 1) * (kC / 2); c += 4) {
-              float2 x0 = ptx::fma2(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2);
-              float2 x1 = ptx::fma2(make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, nm2);
+                for (int c0 = 0; c0 < D; c0 += 32) {
+                  uint32_t r[32];
+                  ptx::tmem_ld32(tO + c0, r);
+                  ptx::tmem_wait_ld();
+#pragma unroll
+                  for (int c = 0; c < 32; c += 2) {
+                    const float2 v = ptx::mul2(
+                        make_float2(__uint_as_float(r[c]), __uint_as_float(r[c + 1])), a2);
+                    r[c] = __float_as_uint(v.x);
+                    r[c + 1] = __float_as_uint(v.y);
+                  }
+                  ptx::tmem_st32(tO + c0, r);
+                }
+              }
+            }
+            // p = 2^(s * scale_log2 - m_ref), two columns per instruction; the bf16 pairs
+            // overwrite the low half of the register array
+            PT_MARK(3);
+            const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+            const float2 nm2 = make_float2(-m_ref, -m_ref);
+            float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int c = 0; c < 64; c += 4) {
+              float2 x0 = ptx::fma2(
+                  make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2);
+              float2 x1 = ptx::fma2(
+                  make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, nm2);
               x0.x = ptx::ex2_approx(x0.x);
               x0.y = ptx::ex2_approx(x0.y);
               x1.x = ptx::ex2_approx(x1.x);
@@ -562,50 +600,28 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               sr[c >> 1] = ptx::pack_bf16x2(x0.x, x0.y);
               sr[(c >> 1) + 1] = ptx::pack_bf16x2(x1.x, x1.y);
             }
-            if (C::kHasV) {
-              if (kC == 128) ptx::tmem_st32(tS + half * 32, &sr[half * 32]);
-              else ptx::tmem_st16(tS + half * 16, &sr[half * 16]);
-#ifdef LOSA_X_LATE_P0
-              if (half == 1) {
-#else
-              if (half == 0) {
-#endif
-                ptx::tmem_wait_st();
-                ptx::tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&ctl->p_ready[qt][0]);
-              }
-            }
-          }
-          PT_MARK(4);
-          const float tsum = (acc0.x + acc0.y) + (acc1.x + acc1.y);
-          l += tsum;
-          if (!C::kHasV) tab[(int64_t)j * 128] = make_float2(tsum, m_ref);
-        } else if (C::kHasV) {
-          // this half of the 128-row tile does not list the key block: P = 0
-          uint32_t z[32];
+            PT_MARK(4);
+            const float tsum = (acc0.x + acc0.y) + (acc1.x + acc1.y);
+            l += tsum;
+            if (C::kHasV) ptx::tmem_st32(tSb, sr);
+            else tab[((int64_t)j * (kC / 64) + hs) * 128] = make_float2(tsum, m_ref);
+          } else if (C::kHasV) {
+            // this half of the 128-row tile does not list the key block: P = 0
+            uint32_t z[32];
 #pragma unroll
-          for (int c = 0; c < 32; ++c) z[c] = 0u;
-          if (kC == 128) {
-            ptx::tmem_st32(tS, z);
-            ptx::tmem_st32(tS + 32, z);
-          } else {
-            ptx::tmem_st32(tS, z);
+            for (int c = 0; c < 32; ++c) z[c] = 0u;
+            ptx::tmem_st32(tSb, z);
           }
-          ptx::tmem_wait_st();
+          if (C::kHasV) {
+            ptx::tmem_wait_st();
+            ++pv_item;
+          }
           ptx::tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(&ctl->p_ready[qt][0]);
+          if (lane == 0) ptx::mbar_arrive(&ctl->p_ready[qt][buf]);
+          ++nsub;
+          PT_MARK(5);
         }
-        if (C::kHasV) {
-          ptx::tmem_wait_st();
-          ++pv_item;
-        }
-        ptx::tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&ctl->p_ready[qt][C::kHasV ? 1 : 0]);
-
-        PT_MARK(5);
       }
 
       if (MODE != kMass) {
@@ -615,8 +631,10 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const float inv = (l > 0.f) ? 1.f / l : 0.f;
           const int64_t off = (int64_t)b * p.sb + (int64_t)h * p.sh + (int64_t)grow * p.sn;
           if (pv_item > 0) {
-            LOSA_WAIT(&ctl->o_done[qt], npv & 1);
-            ++npv;
+            // o_done advances once per item, so its parity is unambiguous here (pv_done may be
+            // one, two or three phases from this warp's last look at it)
+            LOSA_WAIT(&ctl->o_done[qt], nod & 1);
+            ++nod;
             ptx::tc_fence_after_sync();
           }
 #pragma unroll
@@ -657,7 +675,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
         }
       } else {
-        // ---- epilogue of the mass pass: normalise the per-tile sums by the final row
+        // ---- epilogue of the mass pass: normalise the per-sub-tile sums by the final row
         // statistics and average them over the rows of each query block
         if (T < p.nQt) {
           const bool valid = grow < p.N;
@@ -669,18 +687,22 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         LOSA_WAIT(&ctl->wg_bar[qt], nwg & 1);
         ++nwg;
         if (T < p.nQt) {
-          const float2* tb = p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * 128;
+          const float2* tb =
+              p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * (kC / 64) * 128;
           for (int u = wl; u < p.nKb; u += 4) {
+            const int subs = (u == p.nKb - 1) ? p.tail_subs : (kC / 64);
             float acc[kQBT];
 #pragma unroll
             for (int q = 0; q < kQBT; ++q) acc[q] = 0.f;
+            for (int hs = 0; hs < subs; ++hs) {
 #pragma unroll
-            for (int rr = 0; rr < 4; ++rr) {
-              const int r = rr * 32 + lane;
-              const float2 tv = tb[(int64_t)u * 128 + r];
-              const float2 st = ctl->rowstat[qt][r];
-              const float wgt = (st.y > 0.f) ? tv.x * ptx::ex2_approx(tv.y - st.x) * st.y : 0.f;
-              acc[(rr * 32) / BLK] += wgt;
+              for (int rr = 0; rr < 4; ++rr) {
+                const int r = rr * 32 + lane;
+                const float2 tv = tb[((int64_t)u * (kC / 64) + hs) * 128 + r];
+                const float2 st = ctl->rowstat[qt][r];
+                const float wgt = (st.y > 0.f) ? tv.x * ptx::ex2_approx(tv.y - st.x) * st.y : 0.f;
+                acc[(rr * 32) / BLK] += wgt;
+              }
             }
 #pragma unroll
             for (int q = 0; q < kQBT; ++q) {
@@ -828,7 +850,7 @@ int dispatch(const Geometry& g, const void* q, const void* k, const void* v, con
 
 size_t attn_workspace_bytes(AttnMode mode, const Geometry& g) {
   if (mode != kMass) return 0;
-  return (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2);
+  return (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * (g.C / 64) * 128 * sizeof(float2);
 }
 
 int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, const void* v,
@@ -843,6 +865,7 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
   prm.nQt = g.nQt;
   prm.nPairs = g.nPairs;
   prm.nWork = g.B * g.H * g.nPairs;
+  prm.tail_subs = (g.N - (g.nKb - 1) * g.C + 63) / 64;
   prm.offsets = offsets;
   prm.kv_idx = kv_idx;
   prm.o = o;
