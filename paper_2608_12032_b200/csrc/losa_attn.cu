@@ -43,6 +43,11 @@ static_assert(128 * kRegsUtility + 256 * kRegsSoftmax <= kThreads * kRegsAtLaunc
               "register reallocation exceeds the CTA's launch allocation");
 static_assert(kThreads * kRegsAtLaunch <= 65536, "launch allocation exceeds the register file");
 constexpr int kTmemCols = 512;
+// Tile list ring: the scheduler warp writes one 32-bit entry per work item header, per K/V tile
+// and one end marker; every other warp reads all of them in order.
+constexpr int kTlChunks = 8;
+constexpr uint32_t kTlItem = 1u << 28, kTlEnd = 2u << 28;  // entry type in bits 31:28 (0 = tile)
+constexpr int kTlConsumers = 11;                           // producer, 2 issuers, 8 softmax warps
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;
@@ -59,7 +64,9 @@ struct Cfg {
   static constexpr int kKVBytes = kDH * kKVSlab;      // one K (or V) tile
   static constexpr bool kHasV = (MODE != kMass);
   static constexpr int kRingBudget = (kHasV ? 160 : 128) * 1024;  // K + V rings
-  static constexpr int kNV = kHasV ? ((kKVBytes >= 32768) ? 2 : 4) : 0;
+  // a V tile stays in use about one tile longer than a K tile (its products are issued one
+  // sub-tile behind), so V gets the deeper ring
+  static constexpr int kNV = kHasV ? ((kKVBytes >= 32768) ? 3 : 4) : 0;
   static constexpr int kNK0 = (kRingBudget - kNV * kKVBytes) / kKVBytes;
   static constexpr int kNK = kNK0 > 6 ? 6 : kNK0;
   static constexpr uint32_t kIdescQK = ptx::idesc_bf16_f32(128, 64, false, false);  // 64-key sub-tile
@@ -89,6 +96,8 @@ struct Control {
   uint64_t s_full[2][2], p_ready[2][2];  // per query tile and S buffer
   uint64_t pv_done[2], o_done[2], o_free[2];  // per product / per item / O read out
   uint64_t wg_bar[2];
+  uint64_t tl_full[kTlChunks], tl_empty[kTlChunks];  // tile list ring, per 32-entry chunk
+  uint32_t tl[kTlChunks * 32];
   uint64_t drain;
   uint32_t tmem_base;
   int abort_flag;
@@ -219,6 +228,34 @@ struct TileIter {
     }                                                            \
   } while (0)
 
+// Next entry of the tile list (whole warp): waits for the chunk when entering it and hands it
+// back to the scheduler after its last entry.  `te` is the warp's running entry counter.
+#define LOSA_TL_NEXT(ent)                                                            \
+  do {                                                                               \
+    const uint32_t c_ = (te >> 5) & (kTlChunks - 1);                                 \
+    if ((te & 31) == 0) LOSA_WAIT(&ctl->tl_full[c_], (te / (kTlChunks * 32)) & 1);   \
+    (ent) = *reinterpret_cast<volatile uint32_t*>(&ctl->tl[te & (kTlChunks * 32 - 1)]); \
+    if ((te & 31) == 31) {                                                           \
+      __syncwarp();                                                                  \
+      if (lane == 0) ptx::mbar_arrive(&ctl->tl_empty[c_]);                           \
+    }                                                                                \
+    ++te;                                                                            \
+  } while (0)
+
+// Scheduler side: append one entry (whole warp; lane 0 writes).
+#define LOSA_TL_PUT(ent)                                                             \
+  do {                                                                               \
+    const uint32_t c_ = (te >> 5) & (kTlChunks - 1);                                 \
+    if ((te & 31) == 0)                                                              \
+      LOSA_WAIT(&ctl->tl_empty[c_], ((te / (kTlChunks * 32)) & 1) ^ 1);              \
+    if (lane == 0) ctl->tl[te & (kTlChunks * 32 - 1)] = (ent);                       \
+    if ((te & 31) == 31) {                                                           \
+      __syncwarp();                                                                  \
+      if (lane == 0) ptx::mbar_arrive(&ctl->tl_full[c_]);                            \
+    }                                                                                \
+    ++te;                                                                            \
+  } while (0)
+
 template <int D, int BLK, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -259,7 +296,11 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       ptx::mbar_init(&ctl->v_full[i], 1);
       ptx::mbar_init(&ctl->v_empty[i], 2);
     }
-    ptx::mbar_init(&ctl->drain, 1);
+    for (int i = 0; i < kTlChunks; ++i) {
+      ptx::mbar_init(&ctl->tl_full[i], 1);
+      ptx::mbar_init(&ctl->tl_empty[i], kTlConsumers);
+    }
+    ptx::mbar_init(&ctl->drain, 2);  // both MMA issuers arrive on the abort path
     ctl->abort_flag = 0;
     ptx::fence_barrier_init();
   }
@@ -285,9 +326,11 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // ------------------------------------------------------------------ TMA producer
     // (the whole warp walks the tile list; lane 0 alone issues the copies)
     {
-      uint32_t nq[2] = {0, 0}, nk = 0, nv = 0;
+      uint32_t nq[2] = {0, 0}, nk = 0, nv = 0, te = 0, ent;
       PT_DECL();
-      for (int w = blockIdx.x; w < p.nWork; w += gridDim.x) {
+      LOSA_TL_NEXT(ent);
+      while ((ent >> 28) == 1) {
+        const int w = (int)(ent & 0x0fffffffu);
         const int bh = w / p.nPairs, pr = w % p.nPairs;
         const int b = bh / p.H, h = bh % p.H;
 #pragma unroll
@@ -307,11 +350,10 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             ++nq[qt];
           }
         }
-        TileIter<kNB> it;
-        it.init(p, MODE != kSparse, bh, 2 * pr * kQBT, lane);
-        int j;
-        uint32_t memb;
-        while (it.next(j, memb)) {
+        for (;;) {
+          LOSA_TL_NEXT(ent);
+          if ((ent >> 28) != 0) break;
+          const int j = (int)(ent & 0xffffu);
           const uint32_t ks = nk % C::kNK;
           PT_MARK(0);
           LOSA_WAIT(&ctl->k_empty[ks], ((nk / C::kNK) & 1) ^ 1);
@@ -358,7 +400,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const bool leader = (lane == 0);
       const uint32_t q_base = ptx::smem_u32(sQ), k_base = ptx::smem_u32(sK),
                      v_base = ptx::smem_u32(sV);
-      uint32_t nq = 0, nt = 0, nsub = 0, npv = 0, nof = 0;
+      uint32_t nq = 0, nt = 0, nsub = 0, npv = 0, nof = 0, te = 0, ent;
       // nt: tiles walked, nsub: S sub-tiles issued, npv: P V products issued (kernel lifetime)
       PT_DECL();
 
@@ -424,15 +466,15 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     PT_MARK(6);                                                                    \
   } while (0)
 
-      for (int w = blockIdx.x; w < p.nWork; w += gridDim.x) {
-        const int bh = w / p.nPairs, pr = w % p.nPairs;
-        TileIter<kNB> it;
-        it.init(p, MODE != kSparse, bh, 2 * pr * kQBT, lane);
+      LOSA_TL_NEXT(ent);
+      while ((ent >> 28) == 1) {
         bool q_ready = false;
         pv_item = 0;
-        int j;
-        uint32_t memb;
-        while (it.next(j, memb)) {
+        for (;;) {
+          LOSA_TL_NEXT(ent);
+          if ((ent >> 28) != 0) break;
+          const int j = (int)(ent & 0xffffu);
+          const uint32_t memb = (ent >> 16) & 0xfu;
           const uint32_t ks = nt % C::kNK, kph = (nt / C::kNK) & 1;
           const uint32_t vs = nt % kNVs, vph = (nt / kNVs) & 1;
           const bool member = ((memb >> (qt * kQBT)) & kQMask) != 0;
@@ -486,6 +528,25 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       PT_MARK(0);
       if (qt == 0) PT_FLUSH(3);
     }
+  } else {
+    // ------------------------------------------------------------------ scheduler (warp 11)
+    // Walks the block-index lists of this CTA's work items and publishes, per item, a header
+    // and the ascending merge of its tiles; nobody else touches the CSR.
+    uint32_t te = 0;
+    for (int w = blockIdx.x; w < p.nWork; w += gridDim.x) {
+      const int bh = w / p.nPairs, pr = w % p.nPairs;
+      LOSA_TL_PUT(kTlItem | (uint32_t)w);
+      TileIter<kNB> it;
+      it.init(p, MODE != kSparse, bh, 2 * pr * kQBT, lane);
+      int j;
+      uint32_t memb;
+      while (it.next(j, memb)) LOSA_TL_PUT((uint32_t)j | (memb << 16));
+    }
+    LOSA_TL_PUT(kTlEnd);
+    if ((te & 31) != 0) {  // publish the last, partly filled chunk
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&ctl->tl_full[((te - 1) >> 5) & (kTlChunks - 1)]);
+    }
   }
   } else {
     // ------------------------------------------------------------------ softmax warpgroups
@@ -499,23 +560,26 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int my_bit = qt * kQBT + sub;
     const int tail = p.N - (p.nKb - 1) * kC;  // valid keys of the last K/V tile
     uint32_t nsub = 0, nwg = 0, nod = 0;      // nsub: sub-tiles of this query tile so far
+    uint32_t te = 0, ent;
     PT_DECL();
 
-    for (int w = blockIdx.x; w < p.nWork; w += gridDim.x) {
+    LOSA_TL_NEXT(ent);
+    while ((ent >> 28) == 1) {
+      const int w = (int)(ent & 0x0fffffffu);
       const int bh = w / p.nPairs, pr = w % p.nPairs;
       const int b = bh / p.H, h = bh % p.H;
       const int T = 2 * pr + qt;
       const int grow = T * 128 + row;
-      TileIter<kNB> it;
-      it.init(p, MODE != kSparse, bh, 2 * pr * kQBT, lane);
       float m_ref = -INFINITY, l = 0.f;
       uint32_t pv_item = 0;
       float2* tab = nullptr;
       if (MODE == kMass)
         tab = p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * (kC / 64) * 128 + row;
-      int j;
-      uint32_t memb;
-      while (it.next(j, memb)) {
+      for (;;) {
+        LOSA_TL_NEXT(ent);
+        if ((ent >> 28) != 0) break;
+        const int j = (int)(ent & 0xffffu);
+        const uint32_t memb = (ent >> 16) & 0xfu;
         if (((memb >> (qt * kQBT)) & kQMask) == 0) continue;
         const bool mine = (memb >> my_bit) & 1u;
         const int subs = (j == p.nKb - 1) ? p.tail_subs : (kC / 64);
@@ -749,6 +813,8 @@ teardown:
   }
 }
 
+#undef LOSA_TL_NEXT
+#undef LOSA_TL_PUT
 #undef LOSA_WAIT
 
 // ---------------------------------------------------------------------------- host side
