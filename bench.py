@@ -279,6 +279,8 @@ def main():
     kv_idx = torch.empty(rows * nKb, dtype=torch.int32, device=dev)
     ws_sel = torch.empty(max(1, losa.binding._select_workspace_bytes(wl.B, wl.H, wl.nQb, nKb)),
                          dtype=torch.uint8, device=dev)
+    ws_attn = torch.empty(max(losa.losa_workspace_bytes(2, prob), losa.losa_workspace_bytes(3, prob)),
+                          dtype=torch.uint8, device=dev)
     o_sparse = torch.empty_like(draws[0][0])
     o_dense = torch.empty_like(draws[0][0])
 
@@ -293,10 +295,10 @@ def main():
         losa.losa_select(mass, tau, ws=ws_sel, out=(offsets, kv_idx))
         marks.append(ev()); marks[-1].record()
         for (q, k, v) in draws:
-            losa.losa_sparse_attn(q, k, v, offsets, kv_idx, wl.R, wl.C, out=o_sparse)
+            losa.losa_sparse_attn(q, k, v, offsets, kv_idx, wl.R, wl.C, out=o_sparse, ws=ws_attn)
             marks.append(ev()); marks[-1].record()
         q, k, v = draws[0]
-        losa.losa_attn(q, k, v, wl.R, wl.C, out=o_dense)
+        losa.losa_attn(q, k, v, wl.R, wl.C, out=o_dense, ws=ws_attn)
         marks.append(ev()); marks[-1].record()
         if record is not None:
             record.append(marks)
@@ -360,7 +362,7 @@ def main():
                 qd.copy_(q, non_blocking=True)
                 kd.copy_(k, non_blocking=True)
                 vd.copy_(v, non_blocking=True)
-                losa.losa_sparse_attn(qd, kd, vd, offsets, kv_idx, wl.R, wl.C, out=o_sparse)
+                losa.losa_sparse_attn(qd, kd, vd, offsets, kv_idx, wl.R, wl.C, out=o_sparse, ws=ws_attn)
                 o_host.copy_(o_sparse, non_blocking=True)
 
         e2e_step()

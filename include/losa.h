@@ -69,8 +69,8 @@ typedef struct {
 } losa_problem_t;
 
 /* Bytes of caller-provided device workspace an operation needs for this problem
- * (LOSA_OP_*).  For LOSA_OP_SELECT only B, H, N, R, C are read.  Returns 0 for
- * operations that need none, and 0 for an invalid problem.  Host-only: touches no GPU. */
+ * (LOSA_OP_*).  For LOSA_OP_SELECT only B, H, N, R, C are read.  Returns 0 for an invalid
+ * problem.  Host-only: touches no GPU. */
 size_t losa_workspace_bytes(int op, const losa_problem_t* p);
 
 /* Exact block attention mass of one dense attention step (Eq. 1).
@@ -142,14 +142,17 @@ int losa_select_noalloc(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const fl
  *     o(q) = sum_{k in K(q)} softmax_{K(q)}(q k^T * scale) v(k).
  * The CSR must satisfy losa_validate_csr(); a block index outside [0, nKb) is skipped and
  * reported as LOSA_ERR_BAD_INDEX, never dereferenced.
- *   q, k, v  bf16 [B,H,N,D];  o  [B,H,N,D] with the same strides, bf16 or f32 (o_dtype)   */
+ *   q, k, v  bf16 [B,H,N,D];  o  [B,H,N,D] with the same strides, bf16 or f32 (o_dtype)
+ *   ws       >= losa_workspace_bytes(LOSA_OP_SPARSE_ATTN, p) bytes (a few hundred: the
+ *            counter the persistent CTAs draw work items from); not shared between calls
+ *            that may run concurrently                                                    */
 int losa_sparse_attn(const losa_problem_t* p, const void* q, const void* k, const void* v,
                      const int32_t* offsets, const int32_t* kv_idx, void* o, int o_dtype,
                      void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* Dense softmax attention o = softmax(q k^T * scale) v over the N valid keys: the paper's
  * dense steps up to the construction step, and this library's own dense baseline.
- * Same tensors as losa_sparse_attn without the CSR. */
+ * Same tensors and workspace rule as losa_sparse_attn, without the CSR. */
 int losa_attn(const losa_problem_t* p, const void* q, const void* k, const void* v, void* o,
               int o_dtype, void* ws, size_t ws_bytes, void* cuda_stream);
 

@@ -187,26 +187,30 @@ def _select_workspace_bytes(B: int, H: int, nQb: int, nKb: int) -> int:
 
 def losa_sparse_attn(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, offsets: torch.Tensor,
                      kv_idx: torch.Tensor, R: int, C: int, scale: Optional[float] = None,
-                     out_dtype: torch.dtype = torch.bfloat16, out: Optional[torch.Tensor] = None):
+                     out_dtype: torch.dtype = torch.bfloat16, out: Optional[torch.Tensor] = None,
+                     ws: Optional[torch.Tensor] = None):
     """Block-sparse attention over the frozen CSR pattern; rows >= N do not exist."""
     _same_layout(q, k, v)
     prob = make_problem(q, R, C, scale)
     o = _alloc_out(q, out_dtype, out)
+    ws, ws_bytes = _workspace(LOSA_OP_SPARSE_ATTN, prob, q.device, ws)
     _check(_lib().losa_sparse_attn(ctypes.byref(prob), _ptr(q), _ptr(k), _ptr(v), _ptr(offsets),
-                                   _ptr(kv_idx), _ptr(o), _dtype_code(o.dtype), None, 0, _stream()),
+                                   _ptr(kv_idx), _ptr(o), _dtype_code(o.dtype), _ptr(ws), ws_bytes,
+                                   _stream()),
            "losa_sparse_attn")
     return o
 
 
 def losa_attn(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, R: int = 128, C: int = 128,
               scale: Optional[float] = None, out_dtype: torch.dtype = torch.bfloat16,
-              out: Optional[torch.Tensor] = None):
+              out: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None):
     """Dense softmax attention with the library's own kernel."""
     _same_layout(q, k, v)
     prob = make_problem(q, R, C, scale)
     o = _alloc_out(q, out_dtype, out)
+    ws, ws_bytes = _workspace(LOSA_OP_ATTN, prob, q.device, ws)
     _check(_lib().losa_attn(ctypes.byref(prob), _ptr(q), _ptr(k), _ptr(v), _ptr(o),
-                            _dtype_code(o.dtype), None, 0, _stream()), "losa_attn")
+                            _dtype_code(o.dtype), _ptr(ws), ws_bytes, _stream()), "losa_attn")
     return o
 
 

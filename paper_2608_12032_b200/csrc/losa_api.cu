@@ -159,21 +159,23 @@ static int check_attn_args(const losa_problem_t* p, Geometry* g, const void* q, 
 int losa_sparse_attn(const losa_problem_t* p, const void* q, const void* k, const void* v,
                      const int32_t* offsets, const int32_t* kv_idx, void* o, int o_dtype, void* ws,
                      size_t ws_bytes, void* cuda_stream) {
-  (void)ws_bytes;  // this operation needs no workspace (diagnostic builds write timers to ws)
   Geometry g;
   int rc = check_attn_args(p, &g, q, k, v, o, o_dtype);
   if (rc != LOSA_OK) return rc;
   if (!offsets || !kv_idx) return LOSA_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < attn_workspace_bytes(kSparse, g)) return LOSA_ERR_WORKSPACE;
+  if (!aligned16(ws)) return LOSA_ERR_INVALID_ARG;
   return launch_attn(kSparse, g, q, k, v, offsets, kv_idx, o, o_dtype, nullptr, nullptr, ws,
                      static_cast<cudaStream_t>(cuda_stream));
 }
 
 int losa_attn(const losa_problem_t* p, const void* q, const void* k, const void* v, void* o,
               int o_dtype, void* ws, size_t ws_bytes, void* cuda_stream) {
-  (void)ws_bytes;
   Geometry g;
   int rc = check_attn_args(p, &g, q, k, v, o, o_dtype);
   if (rc != LOSA_OK) return rc;
+  if (!ws || ws_bytes < attn_workspace_bytes(kDense, g)) return LOSA_ERR_WORKSPACE;
+  if (!aligned16(ws)) return LOSA_ERR_INVALID_ARG;
   return launch_attn(kDense, g, q, k, v, nullptr, nullptr, o, o_dtype, nullptr, nullptr, ws,
                      static_cast<cudaStream_t>(cuda_stream));
 }

@@ -45,6 +45,7 @@ static_assert(kThreads * kRegsAtLaunch <= 65536, "launch allocation exceeds the 
 constexpr int kTmemCols = 512;
 // Tile list ring: the scheduler warp writes one 32-bit entry per work item header, per K/V tile
 // and one end marker; every other warp reads all of them in order.
+constexpr size_t kCounterBytes = 256;  // head of the workspace: the work-item counter
 constexpr int kTlChunks = 8;
 constexpr uint32_t kTlItem = 1u << 28, kTlEnd = 2u << 28;  // entry type in bits 31:28 (0 = tile)
 constexpr int kTlConsumers = 11;                           // producer, 2 issuers, 8 softmax warps
@@ -83,6 +84,7 @@ struct Params {
   int64_t sb, sh, sn;
   float* mass;
   float* lse;
+  int* work_counter;  // zeroed before the launch; CTAs draw work items from it
   float2* table;  // mass mode: [grid][2][nKb * C/64][128] (sum of p, reference max) per row and sub-tile
   float scale_log2;
   int* status;
@@ -533,7 +535,13 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // Walks the block-index lists of this CTA's work items and publishes, per item, a header
     // and the ascending merge of its tiles; nobody else touches the CSR.
     uint32_t te = 0;
-    for (int w = blockIdx.x; w < p.nWork; w += gridDim.x) {
+    for (;;) {
+      // work items are drawn from a global counter, in head-major order, so that a CTA that
+      // finishes early takes the next item instead of idling at the end of the launch
+      int w = 0;
+      if (lane == 0) w = atomicAdd(p.work_counter, 1);
+      w = __shfl_sync(0xffffffffu, w, 0);
+      if (w >= p.nWork) break;
       const int bh = w / p.nPairs, pr = w % p.nPairs;
       LOSA_TL_PUT(kTlItem | (uint32_t)w);
       TileIter<kNB> it;
@@ -915,8 +923,8 @@ int dispatch(const Geometry& g, const void* q, const void* k, const void* v, con
 }  // namespace
 
 size_t attn_workspace_bytes(AttnMode mode, const Geometry& g) {
-  if (mode != kMass) return 0;
-  return (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * (g.C / 64) * 128 * sizeof(float2);
+  if (mode != kMass) return kCounterBytes;
+  return kCounterBytes + (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * (g.C / 64) * 128 * sizeof(float2);
 }
 
 int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, const void* v,
@@ -941,10 +949,13 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
   prm.sn = g.sn;
   prm.mass = mass;
   prm.lse = lse;
-  prm.table = static_cast<float2*>(ws);
+  // workspace: [0, 256) work counter, then the mass pass's per-CTA table
+  prm.work_counter = static_cast<int*>(ws);
+  prm.table = reinterpret_cast<float2*>(static_cast<char*>(ws) + kCounterBytes);
   prm.scale_log2 = g.scale * kLog2e;
   prm.status = status_word_device();
   if (!prm.status) return LOSA_ERR_CUDA;
+  LOSA_CUDA_TRY(cudaMemsetAsync(prm.work_counter, 0, sizeof(int), st));
   switch (mode) {
     case kDense: return dispatch<kDense>(g, q, k, v, prm, st);
     case kSparse: return dispatch<kSparse>(g, q, k, v, prm, st);
