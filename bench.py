@@ -141,6 +141,20 @@ class ClockSampler:
         }
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def aggregate_tflops(flops_per_call: float, calls: int, slowest_rank_ms: float, world: int) -> float:
+    """Whole-job throughput: every rank does `calls` launches of `flops_per_call`; the job takes as
+    long as its slowest rank (weak scaling, no exchange between ranks)."""
+    return world * flops_per_call * calls / (slowest_rank_ms * 1e-3) / 1e12
+
+
 def cpu_baseline(wl, q, k, v, offsets, kv_idx, seconds: float):
     """The oracle's sparse attention (Eq. 4), as it stands, on a bounded sample of query blocks."""
     from oracle import losa_oracle as orc
@@ -337,13 +351,9 @@ def main():
         dense_ms.append(marks[2 + args.draws].elapsed_time(marks[3 + args.draws]))
     sparse_total_ms = sum(sparse_ms)
 
-    # max over ranks of the times that enter the aggregate
-    t = torch.tensor([total_ms, sparse_total_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms_max, sparse_total_ms_max = (float(x) for x in t.cpu())
+    total_ms_max, sparse_total_ms_max = max_over_ranks([total_ms, sparse_total_ms], dist, dev)
     n_sparse_calls = args.steps * args.draws
-    value = world * flops_sparse * n_sparse_calls / (sparse_total_ms_max * 1e-3) / 1e12
+    value = aggregate_tflops(flops_sparse, n_sparse_calls, sparse_total_ms_max, world)
 
     # ---- end to end through the public API with host buffers (pinned), copies inside the timing
     e2e = None
@@ -374,16 +384,14 @@ def main():
             e2e_step()
         b.record()
         barrier()
-        e2e_ms = torch.tensor([a.elapsed_time(b)], dtype=torch.float64, device=dev)
-        if dist is not None:
-            dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+        (e2e_ms,) = max_over_ranks([a.elapsed_time(b)], dist, dev)
         nbytes = q0.numel() * 2
         e2e = {
-            "value": world * flops_sparse * args.draws * n_e2e / (float(e2e_ms) * 1e-3) / 1e12,
+            "value": aggregate_tflops(flops_sparse, args.draws * n_e2e, e2e_ms, world),
             "unit": UNIT,
             "h2d_bytes_per_step": (2 + 3 * args.draws) * nbytes,
             "d2h_bytes_per_step": args.draws * nbytes,
-            "ms_per_step": float(e2e_ms) / n_e2e,
+            "ms_per_step": e2e_ms / n_e2e,
             "steps": n_e2e,
             "note": "mass+select+draws x sparse attention; every call's q/k/v copied from pinned "
                     "host memory and every output copied back inside the timed region",
