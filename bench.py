@@ -38,6 +38,9 @@ from paper_2608_12032_b200 import inputs  # noqa: E402
 METRIC = "block_sparse_attn_effective_tflops"
 UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one sparse-forward launch, from the ncu capture
+# summarised in profiles/losa_attn_kernel_wan_ncu.md (not re-measured by this script)
+NCU_DRAM_BYTES_PER_LAUNCH = {"wan": 0.304484e9 + 0.083875e9}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -433,7 +436,9 @@ def main():
             "frac_of_burst": achieved / float(peaks["bf16_tflops"]),
             "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS,
             "flops_per_launch": flops_sparse,
-            "traffic": None,
+            "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(wl.name),
+            "traffic_unit": "bytes per launch (DRAM read + write, ncu)",
+            "algorithmic_bytes_per_launch": 4 * q0.numel() * 2,
         },
         "clocks": clocks.summary(),
         "gpu_launches": args.steps * (1 + 3 + args.draws + 1),
