@@ -64,13 +64,17 @@ struct Cfg {
   static constexpr int kKVSlab = kC * 128;            // bytes of a [C][64] bf16 slab
   static constexpr int kKVBytes = kDH * kKVSlab;      // one K (or V) tile
   static constexpr bool kHasV = (MODE != kMass);
+  // Keys per S sub-tile.  With an O accumulator in TMEM there is room for two 64-column S buffers
+  // per query tile; the mass pass has no O and uses two 128-column buffers (full-rate 128-wide MMAs).
+  static constexpr int kW = (!kHasV && kC == 128) ? 128 : 64;
+  static constexpr int kSubs = kC / kW;               // sub-tiles per K/V tile
   static constexpr int kRingBudget = (kHasV ? 160 : 128) * 1024;  // K + V rings
   // a V tile stays in use about one tile longer than a K tile (its products are issued one
   // sub-tile behind), so V gets the deeper ring
   static constexpr int kNV = kHasV ? ((kKVBytes >= 32768) ? 3 : 4) : 0;
   static constexpr int kNK0 = (kRingBudget - kNV * kKVBytes) / kKVBytes;
   static constexpr int kNK = kNK0 > 6 ? 6 : kNK0;
-  static constexpr uint32_t kIdescQK = ptx::idesc_bf16_f32(128, 64, false, false);  // 64-key sub-tile
+  static constexpr uint32_t kIdescQK = ptx::idesc_bf16_f32(128, kW, false, false);  // one sub-tile
   static constexpr uint32_t kIdescPV = ptx::idesc_bf16_f32(128, D, false, true);
 };
 
@@ -85,7 +89,7 @@ struct Params {
   float* mass;
   float* lse;
   int* work_counter;  // zeroed before the launch; CTAs draw work items from it
-  float2* table;  // mass mode: [grid][2][nKb * C/64][128] (sum of p, reference max) per row and sub-tile
+  float2* table;  // mass mode: [grid][2][nKb * sub-tiles][128] (sum of p, reference max) per row and sub-tile
   float scale_log2;
   int* status;
 };
@@ -264,7 +268,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                  const __grid_constant__ CUtensorMap map_v, const Params p) {
   using C = Cfg<D, BLK, MODE>;
   using Ctl = Control<C::kNK, C::kNV, MODE == kMass>;
-  constexpr int kC = C::kC, kQBT = C::kQBT, kNB = C::kNB;
+  constexpr int kC = C::kC, kQBT = C::kQBT, kNB = C::kNB, kW = C::kW, kSubs = C::kSubs;
   constexpr uint32_t kQMask = (1u << kQBT) - 1u;
 
   extern __shared__ uint8_t smem_raw[];
@@ -410,18 +414,18 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const uint32_t q_lo = ptx::smem_desc_lo(q_base, 16) + qt * (C::kQBytes >> 4);
       const uint32_t k_lo = ptx::smem_desc_lo(k_base, 16);
       const uint32_t v_lo = ptx::smem_desc_lo(v_base, C::kKVSlab);
-      const uint32_t tS = tmem_base + qt * 128, tO = tmem_base + 256 + qt * 128;
+      const uint32_t tS = tmem_base + qt * 2 * kW, tO = tmem_base + 256 + qt * 128;
       constexpr uint32_t kNVs = C::kNV > 0 ? C::kNV : 1;
 
-      // S[buf] = Q K(stage ks, keys 64 h .. 64 h + 63)^T
+      // S[buf] = Q K(stage ks, sub-tile h)^T
       auto issue_qk = [&](uint32_t ks, int h, uint32_t buf) {
         if (!leader) return;
-        const uint32_t b0 = k_lo + ks * (C::kKVBytes >> 4) + ((h * 64 * 128) >> 4);
+        const uint32_t b0 = k_lo + ks * (C::kKVBytes >> 4) + ((h * kW * 128) >> 4);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t a_off = ((kk >> 2) * C::kQSlab + (kk & 3) * 32) >> 4;
           const uint32_t b_off = ((kk >> 2) * C::kKVSlab + (kk & 3) * 32) >> 4;
-          ptx::mma_ss_lohi(tS + buf * 64, q_lo + a_off, b0 + b_off, kDescHi, C::kIdescQK,
+          ptx::mma_ss_lohi(tS + buf * kW, q_lo + a_off, b0 + b_off, kDescHi, C::kIdescQK,
                            kk > 0 ? 1u : 0u);
         }
       };
@@ -480,7 +484,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const uint32_t ks = nt % C::kNK, kph = (nt / C::kNK) & 1;
           const uint32_t vs = nt % kNVs, vph = (nt / kNVs) & 1;
           const bool member = ((memb >> (qt * kQBT)) & kQMask) != 0;
-          const int subs = (j == p.nKb - 1) ? p.tail_subs : (kC / 64);
+          const int subs = (j == p.nKb - 1) ? p.tail_subs : kSubs;
           PT_MARK(0);
           LOSA_WAIT(&ctl->k_full[ks], kph);
           PT_MARK(1);
@@ -562,7 +566,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int qt = warp >> 2, wl = warp & 3;
     const int row = wl * 32 + lane;
     const uint32_t lane_base = (uint32_t)(wl * 32) << 16;
-    const uint32_t tS = tmem_base + lane_base + qt * 128;
+    const uint32_t tS = tmem_base + lane_base + qt * 2 * kW;
     const uint32_t tO = tmem_base + lane_base + 256 + qt * 128;
     const int sub = (BLK == 64) ? (wl >> 1) : 0;
     const int my_bit = qt * kQBT + sub;
@@ -582,7 +586,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       uint32_t pv_item = 0;
       float2* tab = nullptr;
       if (MODE == kMass)
-        tab = p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * (kC / 64) * 128 + row;
+        tab = p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * kSubs * 128 + row;
       for (;;) {
         LOSA_TL_NEXT(ent);
         if ((ent >> 28) != 0) break;
@@ -590,39 +594,39 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint32_t memb = (ent >> 16) & 0xfu;
         if (((memb >> (qt * kQBT)) & kQMask) == 0) continue;
         const bool mine = (memb >> my_bit) & 1u;
-        const int subs = (j == p.nKb - 1) ? p.tail_subs : (kC / 64);
+        const int subs = (j == p.nKb - 1) ? p.tail_subs : kSubs;
         for (int hs = 0; hs < subs; ++hs) {
           const uint32_t buf = nsub & 1, ph = (nsub >> 1) & 1;
-          const uint32_t tSb = tS + buf * 64;
+          const uint32_t tSb = tS + buf * kW;
           PT_MARK(0);
           LOSA_WAIT(&ctl->s_full[qt][buf], ph);
           PT_MARK(1);
           ptx::tc_fence_after_sync();
           if (mine) {
-            uint32_t sr[64];
-            ptx::tmem_ld32(tSb, &sr[0]);
-            ptx::tmem_ld32(tSb + 32, &sr[32]);
+            uint32_t sr[kW];
+#pragma unroll
+            for (int c0 = 0; c0 < kW; c0 += 32) ptx::tmem_ld32(tSb + c0, &sr[c0]);
             ptx::tmem_wait_ld();
             PT_MARK(2);
             if (j == p.nKb - 1) {
-              const int valid = tail - hs * 64;  // keys >= N do not exist
-              if (valid < 64) {
+              const int valid = tail - hs * kW;  // keys >= N do not exist
+              if (valid < kW) {
 #pragma unroll
-                for (int c = 0; c < 64; ++c)
+                for (int c = 0; c < kW; ++c)
                   if (c >= valid) sr[c] = 0xff800000u;
               }
             }
             float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
             float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
 #pragma unroll
-            for (int c = 4; c + 8 <= 64; c += 8) {
+            for (int c = 4; c + 8 <= kW; c += 8) {
               mx0 = ptx::max3(mx0, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
               mx1 = ptx::max3(mx1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
               mx2 = ptx::max3(mx2, __uint_as_float(sr[c + 4]), __uint_as_float(sr[c + 5]));
               mx3 = ptx::max3(mx3, __uint_as_float(sr[c + 6]), __uint_as_float(sr[c + 7]));
             }
-            mx0 = ptx::max3(mx0, __uint_as_float(sr[60]), __uint_as_float(sr[61]));
-            mx1 = ptx::max3(mx1, __uint_as_float(sr[62]), __uint_as_float(sr[63]));
+            mx0 = ptx::max3(mx0, __uint_as_float(sr[kW - 4]), __uint_as_float(sr[kW - 3]));
+            mx1 = ptx::max3(mx1, __uint_as_float(sr[kW - 2]), __uint_as_float(sr[kW - 1]));
             const float m_new =
                 fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
             const bool need = m_new > m_ref + kRescaleThreshold;
@@ -658,7 +662,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const float2 nm2 = make_float2(-m_ref, -m_ref);
             float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
 #pragma unroll
-            for (int c = 0; c < 64; c += 4) {
+            for (int c = 0; c < kW; c += 4) {
               float2 x0 = ptx::fma2(
                   make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2);
               float2 x1 = ptx::fma2(
@@ -676,7 +680,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const float tsum = (acc0.x + acc0.y) + (acc1.x + acc1.y);
             l += tsum;
             if (C::kHasV) ptx::tmem_st32(tSb, sr);
-            else tab[((int64_t)j * (kC / 64) + hs) * 128] = make_float2(tsum, m_ref);
+            else tab[((int64_t)j * kSubs + hs) * 128] = make_float2(tsum, m_ref);
           } else if (C::kHasV) {
             // this half of the 128-row tile does not list the key block: P = 0
             uint32_t z[32];
@@ -760,9 +764,9 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         ++nwg;
         if (T < p.nQt) {
           const float2* tb =
-              p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * (kC / 64) * 128;
+              p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * kSubs * 128;
           for (int u = wl; u < p.nKb; u += 4) {
-            const int subs = (u == p.nKb - 1) ? p.tail_subs : (kC / 64);
+            const int subs = (u == p.nKb - 1) ? p.tail_subs : kSubs;
             float acc[kQBT];
 #pragma unroll
             for (int q = 0; q < kQBT; ++q) acc[q] = 0.f;
@@ -770,7 +774,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
               for (int rr = 0; rr < 4; ++rr) {
                 const int r = rr * 32 + lane;
-                const float2 tv = tb[((int64_t)u * (kC / 64) + hs) * 128 + r];
+                const float2 tv = tb[((int64_t)u * kSubs + hs) * 128 + r];
                 const float2 st = ctl->rowstat[qt][r];
                 const float wgt = (st.y > 0.f) ? tv.x * ptx::ex2_approx(tv.y - st.x) * st.y : 0.f;
                 acc[(rr * 32) / BLK] += wgt;
@@ -924,7 +928,8 @@ int dispatch(const Geometry& g, const void* q, const void* k, const void* v, con
 
 size_t attn_workspace_bytes(AttnMode mode, const Geometry& g) {
   if (mode != kMass) return kCounterBytes;
-  return kCounterBytes + (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * (g.C / 64) * 128 * sizeof(float2);
+  // the mass pass uses one sub-tile per key tile at both supported block sizes
+  return kCounterBytes + (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2);
 }
 
 int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, const void* v,
@@ -939,7 +944,8 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
   prm.nQt = g.nQt;
   prm.nPairs = g.nPairs;
   prm.nWork = g.B * g.H * g.nPairs;
-  prm.tail_subs = (g.N - (g.nKb - 1) * g.C + 63) / 64;
+  const int sub_w = (mode == kMass && g.C == 128) ? 128 : 64;  // Cfg::kW
+  prm.tail_subs = (g.N - (g.nKb - 1) * g.C + sub_w - 1) / sub_w;
   prm.offsets = offsets;
   prm.kv_idx = kv_idx;
   prm.o = o;

@@ -57,18 +57,18 @@ select_rows_kernel(const float* __restrict__ mass, int nKb, int n2, double tau,
   if (bad) report_error(status, LOSA_ERR_BAD_MASS);
   __syncthreads();
 
-  // bitonic sort, ascending keys = descending mass, ties by ascending block index
+  // bitonic sort, ascending keys = descending mass, ties by ascending block index; every thread
+  // owns compare-exchange pairs (i, i | j), so no thread idles
   for (int k = 2; k <= n2; k <<= 1) {
     for (int j = k >> 1; j > 0; j >>= 1) {
-      for (int i = tid; i < n2; i += kSelThreads) {
-        const int ixj = i ^ j;
-        if (ixj > i) {
-          const unsigned long long a = keys[i], b = keys[ixj];
-          const bool up = ((i & k) == 0);
-          if ((a > b) == up) {
-            keys[i] = b;
-            keys[ixj] = a;
-          }
+      for (int pr = tid; pr < (n2 >> 1); pr += kSelThreads) {
+        const int i = ((pr & ~(j - 1)) << 1) | (pr & (j - 1));
+        const int ixj = i | j;
+        const unsigned long long a = keys[i], b = keys[ixj];
+        const bool up = ((i & k) == 0);
+        if ((a > b) == up) {
+          keys[i] = b;
+          keys[ixj] = a;
         }
       }
       __syncthreads();
