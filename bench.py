@@ -6,6 +6,7 @@ One "step" is one pass of the whole path over one synthetic attention layer:
     losa_block_mass(q0, k0) -> losa_select(mass, tau)           (one-time construction)
     losa_sparse_attn(q_t, k_t, v_t, CSR) for t = 1..draws        (frozen pattern, later steps)
     losa_attn(q_1, k_1, v_1)                                     (own dense forward, for the ratio)
+    losa_attn_mass(q_1, k_1, v_1)                                (construction step as one kernel)
 
 The headline value is the effective TFLOP/s of the block-sparse forward, counting the flops of
 the retained blocks only.  Everything is timed with CUDA events on the launching stream.
@@ -298,6 +299,8 @@ def main():
                          dtype=torch.uint8, device=dev)
     ws_attn = torch.empty(max(losa.losa_workspace_bytes(2, prob), losa.losa_workspace_bytes(3, prob)),
                           dtype=torch.uint8, device=dev)
+    ws_fused = torch.empty(losa.losa_workspace_bytes(4, prob), dtype=torch.uint8, device=dev)
+    mass_fused = torch.empty_like(mass)
     o_sparse = torch.empty_like(draws[0][0])
     o_dense = torch.empty_like(draws[0][0])
 
@@ -316,6 +319,8 @@ def main():
             marks.append(ev()); marks[-1].record()
         q, k, v = draws[0]
         losa.losa_attn(q, k, v, wl.R, wl.C, out=o_dense, ws=ws_attn)
+        marks.append(ev()); marks[-1].record()
+        losa.losa_attn_mass(q, k, v, wl.R, wl.C, out=o_dense, mass=mass_fused, ws=ws_fused)
         marks.append(ev()); marks[-1].record()
         if record is not None:
             record.append(marks)
@@ -345,13 +350,14 @@ def main():
     losa.check_async("timed region")
     total_ms = t_start.elapsed_time(t_end)
 
-    mass_ms, sel_ms, sparse_ms, dense_ms = [], [], [], []
+    mass_ms, sel_ms, sparse_ms, dense_ms, fused_ms = [], [], [], [], []
     for marks in records:
         mass_ms.append(marks[0].elapsed_time(marks[1]))
         sel_ms.append(marks[1].elapsed_time(marks[2]))
         for i in range(args.draws):
             sparse_ms.append(marks[2 + i].elapsed_time(marks[3 + i]))
         dense_ms.append(marks[2 + args.draws].elapsed_time(marks[3 + args.draws]))
+        fused_ms.append(marks[3 + args.draws].elapsed_time(marks[4 + args.draws]))
     sparse_total_ms = sum(sparse_ms)
 
     total_ms_max, sparse_total_ms_max = max_over_ranks([total_ms, sparse_total_ms], dist, dev)
@@ -417,7 +423,7 @@ def main():
         "config": {
             "workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "D": wl.D, "R": wl.R, "C": wl.C,
             "tau": tau, "draws": args.draws, "coverage": coverage, "nnz": int(off_h[-1]),
-            "step": "block_mass + select + draws x sparse_attn + 1 dense attn",
+            "step": "block_mass + select + draws x sparse_attn + 1 dense attn + 1 fused attn_mass",
             "l2": "inputs larger than L2: each sparse call reads a different 300 MB draw",
             "pe_base": wl.pe_base, "pe_scale": wl.pe_scale,
         },
@@ -425,6 +431,7 @@ def main():
             "sparse_attn": sparse_avg_ms, "sparse_attn_min": min(sparse_ms),
             "dense_attn": statistics.mean(dense_ms), "block_mass": statistics.mean(mass_ms),
             "select": statistics.mean(sel_ms),
+            "attn_mass_fused": statistics.mean(fused_ms),
         },
         "sparse_vs_dense_speedup": statistics.mean(dense_ms) / sparse_avg_ms,
         "dense_tflops": dense_flops / (statistics.mean(dense_ms) * 1e-3) / 1e12,
@@ -441,7 +448,7 @@ def main():
             "algorithmic_bytes_per_launch": 4 * q0.numel() * 2,
         },
         "clocks": clocks.summary(),
-        "gpu_launches": args.steps * (1 + 3 + args.draws + 1),
+        "gpu_launches": args.steps * (1 + 3 + args.draws + 1 + 1),
     }
     if e2e is not None:
         line["e2e"] = e2e

@@ -12,6 +12,7 @@
  *     losa_sparse_attn  Eq. 4   q, k, v, CSR    -> o
  *     losa_attn         dense softmax attention (the warm-up steps and the
  *                       denominator of the sparse-versus-dense ratio)
+ *     losa_attn_mass    dense attention + block mass in one pass (the construction step)
  *
  * Conventions shared by every call
  * --------------------------------
@@ -57,7 +58,13 @@ enum {
   LOSA_ERR_BAD_MASS = -8     /* negative or NaN mass seen by losa_select (device-side)       */
 };
 
-enum { LOSA_OP_BLOCK_MASS = 0, LOSA_OP_SELECT = 1, LOSA_OP_SPARSE_ATTN = 2, LOSA_OP_ATTN = 3 };
+enum {
+  LOSA_OP_BLOCK_MASS = 0,
+  LOSA_OP_SELECT = 1,
+  LOSA_OP_SPARSE_ATTN = 2,
+  LOSA_OP_ATTN = 3,
+  LOSA_OP_ATTN_MASS = 4
+};
 
 enum { LOSA_DTYPE_BF16 = 0, LOSA_DTYPE_F32 = 1 };
 
@@ -155,6 +162,17 @@ int losa_sparse_attn(const losa_problem_t* p, const void* q, const void* k, cons
  * Same tensors and workspace rule as losa_sparse_attn, without the CSR. */
 int losa_attn(const losa_problem_t* p, const void* q, const void* k, const void* v, void* o,
               int o_dtype, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* The construction step as one kernel: dense attention that also accumulates the exact block
+ * masses (the paper's implementation builds the pattern with "a custom dense-attention kernel
+ * that accumulates exact block masses while computing full attention", Implementation
+ * paragraph; pattern construction coincides with the dense step t0).  Results are those of
+ * losa_attn (o) and losa_block_mass (mass, optional lse) on the same inputs, from one pass over
+ * Q K^T.
+ *   ws   >= losa_workspace_bytes(LOSA_OP_ATTN_MASS, p) bytes                               */
+int losa_attn_mass(const losa_problem_t* p, const void* q, const void* k, const void* v, void* o,
+                   int o_dtype, float* mass, float* lse, void* ws, size_t ws_bytes,
+                   void* cuda_stream);
 
 /* Checks a CSR on the device: offsets[0] == 0, offsets non-decreasing with every row
  * holding between 1 and nKb entries (Eq. 3 keeps at least one block), indices in

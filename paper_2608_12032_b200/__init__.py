@@ -8,6 +8,7 @@ from .binding import (  # noqa: F401
     check_async,
     losa_async_status,
     losa_attn,
+    losa_attn_mass,
     losa_block_mass,
     losa_select,
     losa_select_noalloc,

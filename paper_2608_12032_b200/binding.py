@@ -16,11 +16,12 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "liblosa.so")
 
-LOSA_OP_BLOCK_MASS, LOSA_OP_SELECT, LOSA_OP_SPARSE_ATTN, LOSA_OP_ATTN = 0, 1, 2, 3
+LOSA_OP_BLOCK_MASS, LOSA_OP_SELECT, LOSA_OP_SPARSE_ATTN, LOSA_OP_ATTN, LOSA_OP_ATTN_MASS = 0, 1, 2, 3, 4
 LOSA_DTYPE_BF16, LOSA_DTYPE_F32 = 0, 1
 
 EXPORTS = (
     "losa_workspace_bytes", "losa_block_mass", "losa_select", "losa_sparse_attn", "losa_attn",
+    "losa_attn_mass",
     "losa_select_noalloc", "losa_validate_csr", "losa_async_status", "losa_status_string", "losa_last_cuda_error",
 )
 
@@ -69,6 +70,8 @@ def _lib():
         lib.losa_sparse_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, ctypes.c_int, vp, sz, vp]
         lib.losa_attn.restype = ctypes.c_int
         lib.losa_attn.argtypes = [pp, vp, vp, vp, vp, ctypes.c_int, vp, sz, vp]
+        lib.losa_attn_mass.restype = ctypes.c_int
+        lib.losa_attn_mass.argtypes = [pp, vp, vp, vp, vp, ctypes.c_int, vp, vp, vp, sz, vp]
         lib.losa_validate_csr.restype = ctypes.c_int
         lib.losa_validate_csr.argtypes = [i32, i32, vp, vp, vp]
         lib.losa_async_status.restype = ctypes.c_int
@@ -212,6 +215,25 @@ def losa_attn(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, R: int = 128, C
     _check(_lib().losa_attn(ctypes.byref(prob), _ptr(q), _ptr(k), _ptr(v), _ptr(o),
                             _dtype_code(o.dtype), _ptr(ws), ws_bytes, _stream()), "losa_attn")
     return o
+
+
+def losa_attn_mass(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, R: int, C: int,
+                   scale: Optional[float] = None, out_dtype: torch.dtype = torch.bfloat16,
+                   return_lse: bool = False, out: Optional[torch.Tensor] = None,
+                   mass: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None):
+    """The construction step in one kernel: (o, mass[, lse]) = dense attention + block masses."""
+    _same_layout(q, k, v)
+    prob = make_problem(q, R, C, scale)
+    B, H, N, _ = q.shape
+    o = _alloc_out(q, out_dtype, out)
+    if mass is None:
+        mass = torch.empty((B, H, -(-N // R), -(-N // C)), dtype=torch.float32, device=q.device)
+    lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if return_lse else None
+    ws, ws_bytes = _workspace(LOSA_OP_ATTN_MASS, prob, q.device, ws)
+    _check(_lib().losa_attn_mass(ctypes.byref(prob), _ptr(q), _ptr(k), _ptr(v), _ptr(o),
+                                 _dtype_code(o.dtype), _ptr(mass), _ptr(lse), _ptr(ws), ws_bytes,
+                                 _stream()), "losa_attn_mass")
+    return (o, mass, lse) if return_lse else (o, mass)
 
 
 def losa_validate_csr(offsets: torch.Tensor, kv_idx: torch.Tensor, nKb: int) -> None:

@@ -92,6 +92,7 @@ size_t losa_workspace_bytes(int op, const losa_problem_t* p) {
     case LOSA_OP_BLOCK_MASS: return attn_workspace_bytes(kMass, g);
     case LOSA_OP_SPARSE_ATTN: return attn_workspace_bytes(kSparse, g);
     case LOSA_OP_ATTN: return attn_workspace_bytes(kDense, g);
+    case LOSA_OP_ATTN_MASS: return attn_workspace_bytes(kFused, g);
   }
   return 0;
 }
@@ -177,6 +178,19 @@ int losa_attn(const losa_problem_t* p, const void* q, const void* k, const void*
   if (!ws || ws_bytes < attn_workspace_bytes(kDense, g)) return LOSA_ERR_WORKSPACE;
   if (!aligned16(ws)) return LOSA_ERR_INVALID_ARG;
   return launch_attn(kDense, g, q, k, v, nullptr, nullptr, o, o_dtype, nullptr, nullptr, ws,
+                     static_cast<cudaStream_t>(cuda_stream));
+}
+
+int losa_attn_mass(const losa_problem_t* p, const void* q, const void* k, const void* v, void* o,
+                   int o_dtype, float* mass, float* lse, void* ws, size_t ws_bytes,
+                   void* cuda_stream) {
+  Geometry g;
+  int rc = check_attn_args(p, &g, q, k, v, o, o_dtype);
+  if (rc != LOSA_OK) return rc;
+  if (!mass || !aligned16(mass)) return LOSA_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < attn_workspace_bytes(kFused, g)) return LOSA_ERR_WORKSPACE;
+  if (!aligned16(ws)) return LOSA_ERR_INVALID_ARG;
+  return launch_attn(kFused, g, q, k, v, nullptr, nullptr, o, o_dtype, mass, lse, ws,
                      static_cast<cudaStream_t>(cuda_stream));
 }
 

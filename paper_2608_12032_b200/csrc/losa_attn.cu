@@ -46,6 +46,7 @@ constexpr int kTmemCols = 512;
 // Tile list ring: the scheduler warp writes one 32-bit entry per work item header, per K/V tile
 // and one end marker; every other warp reads all of them in order.
 constexpr size_t kCounterBytes = 256;  // head of the workspace: the work-item counter
+constexpr size_t kRowstatBytes = (size_t)kMaxPersistentCtas * 2 * 128 * sizeof(float2);
 constexpr int kTlChunks = 8;
 constexpr uint32_t kTlItem = 1u << 28, kTlEnd = 2u << 28;  // entry type in bits 31:28 (0 = tile)
 constexpr int kTlConsumers = 11;                           // producer, 2 issuers, 8 softmax warps
@@ -64,6 +65,7 @@ struct Cfg {
   static constexpr int kKVSlab = kC * 128;            // bytes of a [C][64] bf16 slab
   static constexpr int kKVBytes = kDH * kKVSlab;      // one K (or V) tile
   static constexpr bool kHasV = (MODE != kMass);
+  static constexpr bool kWantMass = (MODE == kMass || MODE == kFused);
   // Keys per S sub-tile.  With an O accumulator in TMEM there is room for two 64-column S buffers
   // per query tile; the mass pass has no O and uses two 128-column buffers (full-rate 128-wide MMAs).
   static constexpr int kW = (!kHasV && kC == 128) ? 128 : 64;
@@ -89,12 +91,13 @@ struct Params {
   float* mass;
   float* lse;
   int* work_counter;  // zeroed before the launch; CTAs draw work items from it
-  float2* table;  // mass mode: [grid][2][nKb * sub-tiles][128] (sum of p, reference max) per row and sub-tile
+  float2* rowstat;  // mass modes: [grid][2][128] final (max, 1/sum) of every row of the item
+  float2* table;  // mass modes: [grid][2][nKb * sub-tiles][128] (sum of p, reference max) per row and sub-tile
   float scale_log2;
   int* status;
 };
 
-template <int NK, int NV, bool MASS>
+template <int NK, int NV>
 struct Control {
   uint64_t q_full[2], q_empty[2];
   uint64_t k_full[NK], k_empty[NK];
@@ -107,7 +110,6 @@ struct Control {
   uint64_t drain;
   uint32_t tmem_base;
   int abort_flag;
-  float2 rowstat[2][MASS ? 128 : 1];  // mass pass: final (max, 1/sum) of every row
 };
 
 // Ascending merge of the block-index lists of the (up to NB) query blocks of a work item.
@@ -214,7 +216,7 @@ struct TileIter {
   } while (0)
 #define PT_FLUSH(role)                                                                   \
   do {                                                                                   \
-    if (MODE != kMass && p.table != nullptr && lane == 0) {                              \
+    if ((MODE == kDense || MODE == kSparse) && p.table != nullptr && lane == 0) {                           \
       long long* dst = reinterpret_cast<long long*>(p.table) + ((int64_t)blockIdx.x * 4 + (role)) * 8; \
       for (int i_ = 0; i_ < 8; ++i_) dst[i_] = pt_[i_];                                  \
     }                                                                                    \
@@ -267,7 +269,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, const Params p) {
   using C = Cfg<D, BLK, MODE>;
-  using Ctl = Control<C::kNK, C::kNV, MODE == kMass>;
+  using Ctl = Control<C::kNK, C::kNV>;
   constexpr int kC = C::kC, kQBT = C::kQBT, kNB = C::kNB, kW = C::kW, kSubs = C::kSubs;
   constexpr uint32_t kQMask = (1u << kQBT) - 1u;
 
@@ -585,7 +587,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       float m_ref = -INFINITY, l = 0.f;
       uint32_t pv_item = 0;
       float2* tab = nullptr;
-      if (MODE == kMass)
+      if (C::kWantMass)
         tab = p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * kSubs * 128 + row;
       for (;;) {
         LOSA_TL_NEXT(ent);
@@ -680,7 +682,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const float tsum = (acc0.x + acc0.y) + (acc1.x + acc1.y);
             l += tsum;
             if (C::kHasV) ptx::tmem_st32(tSb, sr);
-            else tab[((int64_t)j * kSubs + hs) * 128] = make_float2(tsum, m_ref);
+            if (C::kWantMass) tab[((int64_t)j * kSubs + hs) * 128] = make_float2(tsum, m_ref);
           } else if (C::kHasV) {
             // this half of the 128-row tile does not list the key block: P = 0
             uint32_t z[32];
@@ -700,7 +702,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
       }
 
-      if (MODE != kMass) {
+      if (C::kHasV) {
         // ---- epilogue: O / l -> global
         if (T < p.nQt) {
           const bool valid = grow < p.N;
@@ -750,12 +752,14 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             ptx::mbar_arrive(&ctl->o_free[qt]);
           }
         }
-      } else {
+      }
+      if (C::kWantMass) {
         // ---- epilogue of the mass pass: normalise the per-sub-tile sums by the final row
         // statistics and average them over the rows of each query block
+        float2* rs = p.rowstat + ((int64_t)blockIdx.x * 2 + qt) * 128;
         if (T < p.nQt) {
           const bool valid = grow < p.N;
-          ctl->rowstat[qt][row] = make_float2(m_ref, (valid && l > 0.f) ? 1.f / l : 0.f);
+          rs[row] = make_float2(m_ref, (valid && l > 0.f) ? 1.f / l : 0.f);
           if (p.lse != nullptr && valid)
             p.lse[(int64_t)bh * p.N + grow] = (m_ref + log2f(l)) * kLn2;
         }
@@ -765,6 +769,9 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (T < p.nQt) {
           const float2* tb =
               p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * kSubs * 128;
+          float2 st[4];  // this lane's four rows
+#pragma unroll
+          for (int rr = 0; rr < 4; ++rr) st[rr] = rs[rr * 32 + lane];
           for (int u = wl; u < p.nKb; u += 4) {
             const int subs = (u == p.nKb - 1) ? p.tail_subs : kSubs;
             float acc[kQBT];
@@ -775,8 +782,8 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               for (int rr = 0; rr < 4; ++rr) {
                 const int r = rr * 32 + lane;
                 const float2 tv = tb[((int64_t)u * kSubs + hs) * 128 + r];
-                const float2 st = ctl->rowstat[qt][r];
-                const float wgt = (st.y > 0.f) ? tv.x * ptx::ex2_approx(tv.y - st.x) * st.y : 0.f;
+                const float wgt =
+                    (st[rr].y > 0.f) ? tv.x * ptx::ex2_approx(tv.y - st[rr].x) * st[rr].y : 0.f;
                 acc[(rr * 32) / BLK] += wgt;
               }
             }
@@ -885,7 +892,7 @@ template <int D, int BLK, int MODE>
 int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Params prm,
              cudaStream_t st) {
   using C = Cfg<D, BLK, MODE>;
-  using Ctl = Control<C::kNK, C::kNV, MODE == kMass>;
+  using Ctl = Control<C::kNK, C::kNV>;
   CUtensorMap mq, mk, mv;
   int rc;
   if ((rc = make_map(&mq, q, g, 128)) != LOSA_OK) return rc;
@@ -927,9 +934,12 @@ int dispatch(const Geometry& g, const void* q, const void* k, const void* v, con
 }  // namespace
 
 size_t attn_workspace_bytes(AttnMode mode, const Geometry& g) {
-  if (mode != kMass) return kCounterBytes;
-  // the mass pass uses one sub-tile per key tile at both supported block sizes
-  return kCounterBytes + (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2);
+  if (mode == kDense || mode == kSparse) return kCounterBytes;
+  // counter, per-CTA row statistics, per-CTA table of one entry per row and sub-tile; the mass
+  // pass has one sub-tile per key tile, the fused pass C / 64
+  const size_t subs = (mode == kMass) ? 1 : (size_t)g.C / 64;
+  return kCounterBytes + kRowstatBytes +
+         (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * subs * 128 * sizeof(float2);
 }
 
 int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, const void* v,
@@ -955,9 +965,11 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
   prm.sn = g.sn;
   prm.mass = mass;
   prm.lse = lse;
-  // workspace: [0, 256) work counter, then the mass pass's per-CTA table
+  // workspace: [0, 256) work counter, then (mass modes) per-CTA row statistics and tables
   prm.work_counter = static_cast<int*>(ws);
-  prm.table = reinterpret_cast<float2*>(static_cast<char*>(ws) + kCounterBytes);
+  prm.rowstat = reinterpret_cast<float2*>(static_cast<char*>(ws) + kCounterBytes);
+  prm.table = reinterpret_cast<float2*>(static_cast<char*>(ws) + kCounterBytes +
+                                        ((mode == kMass || mode == kFused) ? kRowstatBytes : 0));
   prm.scale_log2 = g.scale * kLog2e;
   prm.status = status_word_device();
   if (!prm.status) return LOSA_ERR_CUDA;
@@ -966,6 +978,7 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
     case kDense: return dispatch<kDense>(g, q, k, v, prm, st);
     case kSparse: return dispatch<kSparse>(g, q, k, v, prm, st);
     case kMass: return dispatch<kMass>(g, q, k, v, prm, st);
+    case kFused: return dispatch<kFused>(g, q, k, v, prm, st);
   }
   return LOSA_ERR_INVALID_ARG;
 }

@@ -56,7 +56,7 @@ int launch_select_noalloc(int rows, int nKb, const float* mass, double tau, int3
 int launch_validate_csr(int rows, int nKb, const int32_t* offsets, const int32_t* kv_idx,
                         cudaStream_t st);
 
-enum AttnMode { kDense = 0, kSparse = 1, kMass = 2 };
+enum AttnMode { kDense = 0, kSparse = 1, kMass = 2, kFused = 3 };  // kFused: dense O and mass
 
 size_t attn_workspace_bytes(AttnMode mode, const Geometry& g);
 int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, const void* v,

@@ -98,6 +98,27 @@ def test_block_mass_matches_oracle(shape):
     assert np.abs(lse.cpu().numpy() - lse_ref).max() <= 1e-3
 
 
+@pytest.mark.parametrize("shape", SHAPES)
+def test_fused_construction_step_matches_oracle_and_the_separate_calls(shape):
+    """losa_attn_mass = dense attention + block masses in one pass (the paper's construction kernel)."""
+    losa = lib()
+    B, H, N, D, BLK = shape
+    q, k, v = make(B, H, N, D, 71, 1.5)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    o, mass, lse = losa.losa_attn_mass(qd, kd, vd, BLK, BLK, out_dtype=torch.float32, return_lse=True)
+    o_sep = losa.losa_attn(qd, kd, vd, BLK, BLK, out_dtype=torch.float32)
+    assert losa.losa_async_status() == 0
+    qn, kn, vn = util.to_np(q), util.to_np(k), util.to_np(v)
+    util.assert_output_close(o, orc.dense_attn(qn, kn, vn), f"fused o {shape}")
+    assert torch.equal(o, o_sep)  # same tiles, same order, same arithmetic
+    ref, ref_lse = orc.block_mass(qn, kn, BLK, BLK, return_lse=True)
+    got = mass.cpu().numpy().reshape(ref.shape).astype(np.float64)
+    assert np.abs(got - ref).max() <= util.MASS_TOL
+    assert np.abs(got.sum(1) - 1.0).max() <= util.MASS_TOL
+    nQb = -(-N // BLK)
+    assert np.abs(lse.cpu().numpy() - ref_lse.reshape(B, H, nQb * BLK)[:, :, :N]).max() <= 1e-3
+
+
 @pytest.mark.parametrize("name,taus", [("tiny", (0.5, 0.75, 0.9, 0.99)), ("small", (0.9, 0.99, 1.0))])
 def test_chain_mass_select_sparse_on_named_workloads(name, taus):
     """mass -> select -> sparse on the generator's tensors: strict selection parity on the GPU's

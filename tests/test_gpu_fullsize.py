@@ -114,6 +114,18 @@ def test_full_size_parity_on_sampled_query_blocks(name, n_sample):
               "sparse_max_abs": sparse_err[0], "sparse_mean_abs": sparse_err[1],
               "dense_max_abs": dense_err[0], "dense_mean_abs": dense_err[1]}
 
+    # ---- the construction step as one kernel (dense O + masses) on the same inputs
+    if name == "wan":
+        o_f, mass_f = losa.losa_attn_mass(qd, kd, vd, wl.R, wl.C, out_dtype=torch.float32)
+        o_d = losa.losa_attn(qd, kd, vd, wl.R, wl.C, out_dtype=torch.float32)
+        losa.check_async("fused construction")
+        assert torch.equal(o_f, o_d)
+        gmf = mass_f.cpu().numpy().reshape(wl.rows, wl.nKb)
+        assert float(np.abs(gmf[ids] - ref_mass).max()) <= util.MASS_TOL
+        assert np.abs(gmf.astype(np.float64).sum(1) - 1.0).max() <= util.MASS_TOL
+        record["fused_mass_max_abs"] = float(np.abs(gmf[ids] - ref_mass).max())
+        del o_f, o_d
+
     # ---- the frozen pattern on a later draw (Wan protocol: indices reused on perturbed Q/K/V)
     if name == "wan":
         q1, k1, v1 = inputs.make_reuse_draw(wl, 1, base=base)
