@@ -227,6 +227,15 @@ struct TileIter {
 #define PT_FLUSH(role) do {} while (0)
 #endif
 
+#define LOSA_WAIT_RELAXED(bar, parity)                                   \
+  do {                                                                   \
+    if (!ptx::mbar_wait_relaxed((bar), (parity), &ctl->abort_flag)) {    \
+      ctl->abort_flag = 1;                                               \
+      report_error(p.status, LOSA_ERR_TIMEOUT);                          \
+      goto teardown;                                                     \
+    }                                                                    \
+  } while (0)
+
 #define LOSA_WAIT(bar, parity)                                   \
   do {                                                           \
     if (!ptx::mbar_wait((bar), (parity), &ctl->abort_flag)) {    \
@@ -255,7 +264,7 @@ struct TileIter {
   do {                                                                               \
     const uint32_t c_ = (te >> 5) & (kTlChunks - 1);                                 \
     if ((te & 31) == 0)                                                              \
-      LOSA_WAIT(&ctl->tl_empty[c_], ((te / (kTlChunks * 32)) & 1) ^ 1);              \
+      LOSA_WAIT_RELAXED(&ctl->tl_empty[c_], ((te / (kTlChunks * 32)) & 1) ^ 1);      \
     if (lane == 0) ctl->tl[te & (kTlChunks * 32 - 1)] = (ent);                       \
     if ((te & 31) == 31) {                                                           \
       __syncwarp();                                                                  \
@@ -346,7 +355,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const int T = 2 * pr + qt;
           if (T < p.nQt) {
             PT_MARK(0);
-            LOSA_WAIT(&ctl->q_empty[qt], (nq[qt] & 1) ^ 1);
+            LOSA_WAIT_RELAXED(&ctl->q_empty[qt], (nq[qt] & 1) ^ 1);
             PT_MARK(1);
             if (lane == 0) {
               ptx::mbar_arrive_expect_tx(&ctl->q_full[qt], C::kQBytes);
@@ -364,7 +373,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const int j = (int)(ent & 0xffffu);
           const uint32_t ks = nk % C::kNK;
           PT_MARK(0);
-          LOSA_WAIT(&ctl->k_empty[ks], ((nk / C::kNK) & 1) ^ 1);
+          LOSA_WAIT_RELAXED(&ctl->k_empty[ks], ((nk / C::kNK) & 1) ^ 1);
           PT_MARK(2);
           if (lane == 0) {
             ptx::mbar_arrive_expect_tx(&ctl->k_full[ks], C::kKVBytes);
@@ -377,7 +386,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if (C::kHasV) {
             const uint32_t vs = nv % (C::kNV > 0 ? C::kNV : 1);
             PT_MARK(0);
-            LOSA_WAIT(&ctl->v_empty[vs], ((nv / (C::kNV > 0 ? C::kNV : 1)) & 1) ^ 1);
+            LOSA_WAIT_RELAXED(&ctl->v_empty[vs], ((nv / (C::kNV > 0 ? C::kNV : 1)) & 1) ^ 1);
             PT_MARK(3);
             if (lane == 0) {
               ptx::mbar_arrive_expect_tx(&ctl->v_full[vs], C::kKVBytes);
@@ -834,6 +843,7 @@ teardown:
 
 #undef LOSA_TL_NEXT
 #undef LOSA_TL_PUT
+#undef LOSA_WAIT_RELAXED
 #undef LOSA_WAIT
 
 // ---------------------------------------------------------------------------- host side

@@ -67,6 +67,21 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
   return false;
 }
 
+// Same bound, but for roles that run far ahead of the data path (copy producer, tile-list
+// scheduler): they sleep between polls from the start, so that their waiting costs neither issue
+// slots nor power that the softmax and MMA warps of the same SM could use.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity,
+                                                  volatile int* abort_flag) {
+  for (uint32_t it = 0; it < (1u << 22); ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (it >= 4) {
+      if ((it & 1023u) == 0 && *abort_flag) return false;
+      __nanosleep(it < 64 ? 64 : 256);
+    }
+  }
+  return false;
+}
+
 // ---------------------------------------------------------------- TMA
 
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
