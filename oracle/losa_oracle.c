@@ -12,6 +12,7 @@
  *   mass     M(i,j) = sum_{q in B^Q_i} sum_{k in B^K_j} A(q,k)            (Eq. 1)
  *            stored divided by the number of valid rows of B^Q_i, so that
  *            sum_j mass(i,j) = 1 and the threshold theta*R of Eq. 3 becomes tau.
+ *   top-k    the k heaviest blocks of every row (the fixed-ratio ablation rule)
  *   select   pi = blocks by decreasing mass (equal masses: lower index first),
  *            s = min{ m >= 1 : sum_{r<=m} mass(pi(r)) >= tau },  Omega = pi(1..s)  (Eq. 3)
  *   sparse   O(q) = sum_{k in K(q)} softmax over K(q) only * V(k),
@@ -235,6 +236,47 @@ int losa_oracle_select(const double* mass, int rows, int nKb, double tau, int32_
       qsort(kr, s, sizeof(int32_t), by_index);
     }
     free(keys);
+  }
+  return 0;
+}
+
+/* Fixed-ratio selection (the paper's ablation, "Retained mass versus fixed-ratio top-k
+ * selection"): every row keeps its k heaviest blocks, equal masses by lower index.
+ *   kept  int32 [rows, k]: the kept block indices of each row in ascending order */
+int losa_oracle_select_topk(const double* mass, int rows, int nKb, int k, int32_t* kept) {
+  if (k < 1 || k > nKb) return -2;
+#pragma omp parallel
+  {
+    mass_key_t* keys = (mass_key_t*)malloc(sizeof(mass_key_t) * nKb);
+#pragma omp for schedule(static)
+    for (int r = 0; r < rows; ++r) {
+      for (int j = 0; j < nKb; ++j) {
+        keys[j].m = mass[(int64_t)r * nKb + j];
+        keys[j].j = j;
+      }
+      qsort(keys, nKb, sizeof(mass_key_t), by_mass_desc_then_index);
+      int32_t* kr = kept + (int64_t)r * k;
+      for (int m = 0; m < k; ++m) kr[m] = keys[m].j;
+      qsort(kr, k, sizeof(int32_t), by_index);
+    }
+    free(keys);
+  }
+  return 0;
+}
+
+/* Retained and total block mass of every row under a CSR pattern (the numerator and
+ * denominator of Recall, Eq. 2, before the sum over heads and query blocks). */
+int losa_oracle_row_recall(const double* mass, int rows, int nKb, const int32_t* offsets,
+                           const int32_t* kv_idx, double* retained, double* total) {
+  for (int r = 0; r < rows; ++r) {
+    double tot = 0.0, ret = 0.0;
+    for (int j = 0; j < nKb; ++j) tot += mass[(int64_t)r * nKb + j];
+    for (int p = offsets[r]; p < offsets[r + 1]; ++p) {
+      if (kv_idx[p] < 0 || kv_idx[p] >= nKb) return -3;
+      ret += mass[(int64_t)r * nKb + kv_idx[p]];
+    }
+    retained[r] = ret;
+    total[r] = tot;
   }
   return 0;
 }

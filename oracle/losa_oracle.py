@@ -177,6 +177,29 @@ def select(mass, tau: float) -> Selection:
     return Selection(order, cum, count, kept, float(tau))
 
 
+def select_topk(mass, k: int):
+    """Fixed-ratio rule of the paper's ablation: (offsets, kv_idx) keeping the k heaviest blocks per row."""
+    m = np.ascontiguousarray(mass, dtype=np.float64)
+    rows, nKb = m.shape
+    kept = np.empty((rows, k), dtype=np.int32)
+    _check(_lib().losa_oracle_select_topk(_ptr(m), rows, nKb, int(k), _ptr(kept)), "select_topk")
+    offsets = (np.arange(rows + 1, dtype=np.int64) * k).astype(np.int32)
+    return offsets, kept.reshape(-1)
+
+
+def row_recall(mass, offsets, kv_idx):
+    """Per row: (retained mass, total mass) under the CSR pattern (Eq. 2 before the outer sums)."""
+    m = np.ascontiguousarray(mass, dtype=np.float64)
+    rows, nKb = m.shape
+    off = np.ascontiguousarray(offsets, dtype=np.int32)
+    idx = np.ascontiguousarray(kv_idx, dtype=np.int32)
+    ret = np.empty(rows, dtype=np.float64)
+    tot = np.empty(rows, dtype=np.float64)
+    _check(_lib().losa_oracle_row_recall(_ptr(m), rows, nKb, _ptr(off), _ptr(idx), _ptr(ret), _ptr(tot)),
+           "row_recall")
+    return ret, tot
+
+
 def sparse_attn(q, k, v, R: int, C: int, offsets, kv_idx, scale: Optional[float] = None,
                 row_ids: Optional[Sequence[int]] = None) -> np.ndarray:
     """Attention restricted to the retained key blocks (Eq. 4): ``[n_rows, R, D]`` fp64."""

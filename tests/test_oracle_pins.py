@@ -230,6 +230,32 @@ def test_select_against_numpy_argsort_cumsum():
     assert np.abs(sel.cum - cum).max() < 1e-15
 
 
+def test_topk_against_numpy_and_heaviest_subset():
+    m = random_mass(12, 11, 21, tail=1.5)
+    m[3, 2] = m[3, 7]  # a tie: the lower index wins when only one of the two fits
+    for k in (1, 4, 11):
+        off, idx = orc.select_topk(m, k)
+        assert list(off) == [r * k for r in range(13)]
+        order = np.argsort(-m, axis=1, kind="stable")[:, :k]
+        assert np.array_equal(idx.reshape(12, k), np.sort(order, axis=1))
+        for r in range(12):
+            best = max(m[r, list(c)].sum() for c in itertools.combinations(range(11), k))
+            assert abs(m[r, idx.reshape(12, k)[r]].sum() - best) < 1e-15
+    with pytest.raises(RuntimeError):
+        orc.select_topk(m, 0)
+
+
+def test_row_recall_against_the_definition():
+    m = random_mass(20, 17, 22)
+    sel = orc.select(m, 0.9)
+    ret, tot = orc.row_recall(m, sel.offsets, sel.kv_idx)
+    for r in range(20):
+        kept = sel.kept[r, : sel.count[r]]
+        assert abs(ret[r] - m[r, kept].sum()) < 1e-15 and abs(tot[r] - m[r].sum()) < 1e-15
+    assert abs(ret.sum() / tot.sum() - orc.recall(m, sel.offsets, sel.kv_idx)) < 1e-15
+    assert np.all(ret >= 0.9 - 1e-12)  # the guarantee of Eq. 3 at the construction step
+
+
 def test_select_rejects_bad_tau():
     with pytest.raises(RuntimeError):
         orc.select(np.ones((1, 2)) / 2, 0.0)
