@@ -110,6 +110,22 @@ int losa_select(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const float* mas
                 int32_t* offsets, int32_t* kv_idx, int64_t kv_capacity, void* ws,
                 size_t ws_bytes, void* cuda_stream);
 
+/* Fixed-ratio selection, the rule the paper's ablation compares Eq. 3 with ("Retained mass versus
+ * fixed-ratio top-k selection"): every row keeps its k heaviest blocks (equal masses: lower block
+ * index first), 1 <= k <= nKb.  Same outputs, workspace and error behaviour as losa_select;
+ * offsets[r] = r * k. */
+int losa_select_topk(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const float* mass, int32_t k,
+                     int32_t* offsets, int32_t* kv_idx, int64_t kv_capacity, void* ws,
+                     size_t ws_bytes, void* cuda_stream);
+
+/* Retained and total block mass of every row under a CSR pattern: the numerator and denominator
+ * of Recall (Eq. 2) before the sums over heads and query blocks, accumulated in fp64.
+ * Recall = sum(retained) / sum(total); Coverage is offsets[rows] / (rows * nKb).
+ *   mass f32 [rows, nKb];  retained, total  f64 [rows] (device).  A block index outside
+ *   [0, nKb) is skipped and reported as LOSA_ERR_BAD_INDEX.  Needs no workspace. */
+int losa_row_recall(int32_t rows, int32_t nKb, const float* mass, const int32_t* offsets,
+                    const int32_t* kv_idx, double* retained, double* total, void* cuda_stream);
+
 /* Bytes of the scratch array built into the library for losa_select_noalloc (per GPU). */
 #define LOSA_SELECT_NOALLOC_MAX_SCRATCH (4u * 1024u * 1024u)
 

@@ -12,6 +12,8 @@ from .binding import (  # noqa: F401
     losa_block_mass,
     losa_select,
     losa_select_noalloc,
+    losa_select_topk,
+    losa_row_recall,
     losa_sparse_attn,
     losa_status_string,
     losa_validate_csr,

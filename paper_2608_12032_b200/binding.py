@@ -21,7 +21,7 @@ LOSA_DTYPE_BF16, LOSA_DTYPE_F32 = 0, 1
 
 EXPORTS = (
     "losa_workspace_bytes", "losa_block_mass", "losa_select", "losa_sparse_attn", "losa_attn",
-    "losa_attn_mass",
+    "losa_attn_mass", "losa_select_topk", "losa_row_recall",
     "losa_select_noalloc", "losa_validate_csr", "losa_async_status", "losa_status_string", "losa_last_cuda_error",
 )
 
@@ -64,6 +64,10 @@ def _lib():
         lib.losa_block_mass.argtypes = [pp, vp, vp, vp, vp, vp, sz, vp]
         lib.losa_select.restype = ctypes.c_int
         lib.losa_select.argtypes = [i32, i32, i32, i32, vp, ctypes.c_double, vp, vp, i64, vp, sz, vp]
+        lib.losa_select_topk.restype = ctypes.c_int
+        lib.losa_select_topk.argtypes = [i32, i32, i32, i32, vp, i32, vp, vp, i64, vp, sz, vp]
+        lib.losa_row_recall.restype = ctypes.c_int
+        lib.losa_row_recall.argtypes = [i32, i32, vp, vp, vp, vp, vp, vp]
         lib.losa_select_noalloc.restype = ctypes.c_int
         lib.losa_select_noalloc.argtypes = [i32, i32, i32, i32, vp, ctypes.c_double, vp, vp, i64, vp, vp]
         lib.losa_sparse_attn.restype = ctypes.c_int
@@ -162,6 +166,34 @@ def losa_select(mass: torch.Tensor, tau: float, kv_capacity: Optional[int] = Non
     _check(_lib().losa_select(B, H, nQb, nKb, _ptr(mass), float(tau), _ptr(offsets), _ptr(kv_idx),
                               cap, _ptr(ws), ws.numel(), _stream()), "losa_select")
     return offsets, kv_idx
+
+
+def losa_select_topk(mass: torch.Tensor, k: int, ws: Optional[torch.Tensor] = None):
+    """Fixed-ratio selection: (offsets, kv_idx) keeping the k heaviest blocks of every row."""
+    if mass.dim() != 4 or not mass.is_contiguous() or mass.dtype != torch.float32:
+        raise ValueError("mass must be a contiguous fp32 [B, H, nQb, nKb] tensor")
+    B, H, nQb, nKb = mass.shape
+    rows = B * H * nQb
+    offsets = torch.empty(rows + 1, dtype=torch.int32, device=mass.device)
+    kv_idx = torch.empty(max(rows * int(k), 1), dtype=torch.int32, device=mass.device)
+    if ws is None:
+        ws = torch.empty(_select_workspace_bytes(B, H, nQb, nKb), dtype=torch.uint8, device=mass.device)
+    _check(_lib().losa_select_topk(B, H, nQb, nKb, _ptr(mass), int(k), _ptr(offsets), _ptr(kv_idx),
+                                   kv_idx.numel(), _ptr(ws), ws.numel(), _stream()), "losa_select_topk")
+    return offsets, kv_idx
+
+
+def losa_row_recall(mass: torch.Tensor, offsets: torch.Tensor, kv_idx: torch.Tensor):
+    """(retained, total) fp64 per row: Recall (Eq. 2) is retained.sum() / total.sum()."""
+    if not mass.is_contiguous() or mass.dtype != torch.float32:
+        raise ValueError("mass must be a contiguous fp32 tensor")
+    nKb = mass.shape[-1]
+    rows = mass.numel() // nKb
+    retained = torch.empty(rows, dtype=torch.float64, device=mass.device)
+    total = torch.empty(rows, dtype=torch.float64, device=mass.device)
+    _check(_lib().losa_row_recall(rows, nKb, _ptr(mass), _ptr(offsets), _ptr(kv_idx), _ptr(retained),
+                                  _ptr(total), _stream()), "losa_row_recall")
+    return retained, total
 
 
 def losa_select_noalloc(mass: torch.Tensor, tau: float, offsets: torch.Tensor, kv_idx: torch.Tensor,

@@ -123,8 +123,31 @@ int losa_select(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const float* mas
   const size_t need = select_workspace_bytes(rows, nKb);
   if (!ws || ws_bytes < need) return LOSA_ERR_WORKSPACE;
   if (!aligned16(ws)) return LOSA_ERR_INVALID_ARG;
-  return launch_select((int)rows, nKb, mass, tau, offsets, kv_idx, kv_capacity, ws,
+  return launch_select((int)rows, nKb, mass, tau, 0, offsets, kv_idx, kv_capacity, ws,
                        static_cast<cudaStream_t>(cuda_stream));
+}
+
+int losa_select_topk(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const float* mass, int32_t k,
+                     int32_t* offsets, int32_t* kv_idx, int64_t kv_capacity, void* ws,
+                     size_t ws_bytes, void* cuda_stream) {
+  if (B <= 0 || H <= 0 || nQb <= 0 || nKb <= 0) return LOSA_ERR_INVALID_ARG;
+  if (k < 1 || k > nKb) return LOSA_ERR_INVALID_ARG;
+  if (!mass || !offsets || !kv_idx || kv_capacity < 0) return LOSA_ERR_INVALID_ARG;
+  const int64_t rows = (int64_t)B * H * nQb;
+  if (rows * nKb > INT32_MAX || nKb > 8192) return LOSA_ERR_UNSUPPORTED;
+  const size_t need = select_workspace_bytes(rows, nKb);
+  if (!ws || ws_bytes < need) return LOSA_ERR_WORKSPACE;
+  if (!aligned16(ws)) return LOSA_ERR_INVALID_ARG;
+  return launch_select((int)rows, nKb, mass, 0.5, k, offsets, kv_idx, kv_capacity, ws,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+int losa_row_recall(int32_t rows, int32_t nKb, const float* mass, const int32_t* offsets,
+                    const int32_t* kv_idx, double* retained, double* total, void* cuda_stream) {
+  if (rows <= 0 || nKb <= 0 || !mass || !offsets || !kv_idx || !retained || !total)
+    return LOSA_ERR_INVALID_ARG;
+  return launch_row_recall(rows, nKb, mass, offsets, kv_idx, retained, total,
+                           static_cast<cudaStream_t>(cuda_stream));
 }
 
 int losa_select_noalloc(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const float* mass,

@@ -47,8 +47,11 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // ---- entry points of the kernel translation units (host launchers) -------------------
 
 size_t select_workspace_bytes(int64_t rows, int nKb);
-int launch_select(int rows, int nKb, const float* mass, double tau, int32_t* offsets,
-                  int32_t* kv_idx, int64_t kv_capacity, void* ws, cudaStream_t st);
+int launch_select(int rows, int nKb, const float* mass, double tau, int fixed_count,
+                  int32_t* offsets, int32_t* kv_idx, int64_t kv_capacity, void* ws,
+                  cudaStream_t st);  // fixed_count > 0: keep that many blocks per row instead
+int launch_row_recall(int rows, int nKb, const float* mass, const int32_t* offsets,
+                      const int32_t* kv_idx, double* retained, double* total, cudaStream_t st);
 size_t select_noalloc_workspace_limit();
 int launch_select_noalloc(int rows, int nKb, const float* mass, double tau, int32_t* offsets,
                           int32_t* kv_idx, int64_t kv_capacity, int32_t* device_status,

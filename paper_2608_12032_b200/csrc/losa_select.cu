@@ -24,7 +24,7 @@ __device__ __forceinline__ double key_mass(unsigned long long key) {
 }
 
 __global__ void __launch_bounds__(kSelThreads)
-select_rows_kernel(const float* __restrict__ mass, int nKb, int n2, double tau,
+select_rows_kernel(const float* __restrict__ mass, int nKb, int n2, double tau, int fixed_count,
                    int32_t* __restrict__ counts, uint32_t* __restrict__ bitmaps, int* status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);
@@ -102,6 +102,7 @@ select_rows_kernel(const float* __restrict__ mass, int nKb, int n2, double tau,
   __syncthreads();
   int s = first_pos;
   if (tau >= 1.0 || s > nKb) s = nKb;
+  if (fixed_count > 0) s = min(fixed_count, nKb);  // fixed-ratio rule: the k heaviest blocks
 
   for (int i = lo; i < hi; ++i) {
     if (i < s) {
@@ -195,6 +196,37 @@ validate_csr_kernel(int rows, int nKb, const int32_t* __restrict__ offsets,
   if (bad) report_error(status, LOSA_ERR_BAD_INDEX);
 }
 
+// Retained and total mass of every row under a CSR pattern (Eq. 2 before the outer sums): one
+// warp per row, fp64 partial sums per lane, shuffle tree.
+__global__ void __launch_bounds__(256)
+row_recall_kernel(const float* __restrict__ mass, int rows, int nKb,
+                  const int32_t* __restrict__ offsets, const int32_t* __restrict__ kv_idx,
+                  double* __restrict__ retained, double* __restrict__ total, int* status) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const float* mrow = mass + row * nKb;
+  double tot = 0.0, ret = 0.0;
+  for (int j = lane; j < nKb; j += 32) tot += (double)mrow[j];
+  const int32_t b = offsets[row], e = offsets[row + 1];
+  bool bad = false;
+  for (int p = b + lane; p < e; p += 32) {
+    const int32_t j = kv_idx[p];
+    if (j < 0 || j >= nKb) bad = true;  // skipped, never used as an address
+    else ret += (double)mrow[j];
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    tot += __shfl_xor_sync(0xffffffffu, tot, d);
+    ret += __shfl_xor_sync(0xffffffffu, ret, d);
+  }
+  if (bad) report_error(status, LOSA_ERR_BAD_INDEX);
+  if (lane == 0) {
+    retained[row] = ret;
+    total[row] = tot;
+  }
+}
+
 int next_pow2(int x) {
   int n = 32;
   while (n < x) n <<= 1;
@@ -210,8 +242,9 @@ size_t select_workspace_bytes(int64_t rows, int nKb) {
   return align_up((size_t)rows * sizeof(int32_t), 256) + (size_t)rows * words * sizeof(uint32_t);
 }
 
-int launch_select(int rows, int nKb, const float* mass, double tau, int32_t* offsets,
-                  int32_t* kv_idx, int64_t kv_capacity, void* ws, cudaStream_t st) {
+int launch_select(int rows, int nKb, const float* mass, double tau, int fixed_count,
+                  int32_t* offsets, int32_t* kv_idx, int64_t kv_capacity, void* ws,
+                  cudaStream_t st) {
   int* status = status_word_device();
   if (!status) return LOSA_ERR_CUDA;
   int32_t* counts = static_cast<int32_t*>(ws);
@@ -224,7 +257,8 @@ int launch_select(int rows, int nKb, const float* mass, double tau, int32_t* off
     LOSA_CUDA_TRY(cudaFuncSetAttribute(select_rows_kernel,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   }
-  select_rows_kernel<<<rows, kSelThreads, smem, st>>>(mass, nKb, n2, tau, counts, bitmaps, status);
+  select_rows_kernel<<<rows, kSelThreads, smem, st>>>(mass, nKb, n2, tau, fixed_count, counts, bitmaps,
+                                                      status);
   scan_counts_kernel<<<1, 1024, 0, st>>>(counts, rows, offsets, kv_capacity, status);
   const int warps_per_cta = 8;
   expand_rows_kernel<<<(rows + warps_per_cta - 1) / warps_per_cta, warps_per_cta * 32, 0, st>>>(
@@ -278,7 +312,8 @@ int launch_select_noalloc(int rows, int nKb, const float* mass, double tau, int3
     LOSA_CUDA_TRY(cudaFuncSetAttribute(select_rows_kernel,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   }
-  select_rows_kernel<<<rows, kSelThreads, smem, st>>>(mass, nKb, n2, tau, counts, bitmaps, status);
+  select_rows_kernel<<<rows, kSelThreads, smem, st>>>(mass, nKb, n2, tau, 0, counts, bitmaps,
+                                                      status);
   scan_counts_kernel<<<1, 1024, 0, st>>>(counts, rows, offsets, kv_capacity, status);
   const int warps_per_cta = 8;
   expand_rows_kernel<<<(rows + warps_per_cta - 1) / warps_per_cta, warps_per_cta * 32, 0, st>>>(
@@ -286,6 +321,16 @@ int launch_select_noalloc(int rows, int nKb, const float* mass, double tau, int3
   LOSA_CUDA_TRY(cudaGetLastError());
   if (device_status)
     LOSA_CUDA_TRY(cudaMemcpyAsync(device_status, status, sizeof(int), cudaMemcpyDeviceToDevice, st));
+  return LOSA_OK;
+}
+
+int launch_row_recall(int rows, int nKb, const float* mass, const int32_t* offsets,
+                      const int32_t* kv_idx, double* retained, double* total, cudaStream_t st) {
+  int* status = status_word_device();
+  if (!status) return LOSA_ERR_CUDA;
+  row_recall_kernel<<<(rows + 7) / 8, 256, 0, st>>>(mass, rows, nKb, offsets, kv_idx, retained,
+                                                    total, status);
+  LOSA_CUDA_TRY(cudaGetLastError());
   return LOSA_OK;
 }
 

@@ -104,6 +104,41 @@ def test_select_host_side_argument_errors():
     assert e.value.code == -3
 
 
+@pytest.mark.parametrize("rows,nKb,k", [(16, 33, 1), (16, 33, 20), (8, 256, 170), (4, 929, 557), (8, 40, 40)])
+def test_topk_selection_bit_exact(rows, nKb, k):
+    losa = lib()
+    m32 = random_mass(rows, nKb, 300 + nKb)
+    m32[1, 2] = m32[1, 5]  # a tie
+    off, idx = losa.losa_select_topk(torch.from_numpy(m32).cuda().reshape(1, 1, rows, nKb), k)
+    assert losa.losa_async_status() == 0
+    ref_off, ref_idx = orc.select_topk(m32.astype(np.float64), k)
+    assert np.array_equal(off.cpu().numpy(), ref_off)
+    assert np.array_equal(idx.cpu().numpy()[: rows * k], ref_idx)
+
+
+def test_row_recall_matches_oracle_and_eq3_guarantee():
+    losa = lib()
+    m32 = random_mass(64, 278, 77)
+    mass = torch.from_numpy(m32).cuda().reshape(1, 2, 32, 278)
+    for tau in (0.9, 0.99):
+        off, idx = losa.losa_select(mass, tau)
+        ret, tot = losa.losa_row_recall(mass, off, idx)
+        assert losa.losa_async_status() == 0
+        off_h = off.cpu().numpy()
+        r_ref, t_ref = orc.row_recall(m32.astype(np.float64), off_h, idx.cpu().numpy()[: off_h[-1]])
+        assert np.abs(ret.cpu().numpy() - r_ref).max() < 1e-12
+        assert np.abs(tot.cpu().numpy() - t_ref).max() < 1e-12
+        assert float(ret.min()) >= tau - 1e-12  # retained mass reaches tau in every row
+    # at equal coverage the retained-mass rule keeps at least as much mass per row as any other set
+    k = 100
+    off_k, idx_k = losa.losa_select_topk(mass, k)
+    ret_k, _ = losa.losa_row_recall(mass, off_k, idx_k)
+    rng_off, rng_idx = util.random_csr(64, 278, 5, k / 278)
+    ret_r, _ = losa.losa_row_recall(mass, torch.from_numpy(rng_off).cuda(), torch.from_numpy(rng_idx).cuda())
+    sizes = np.diff(rng_off)
+    assert np.all(ret_k.cpu().numpy()[sizes <= k] >= ret_r.cpu().numpy()[sizes <= k] - 1e-12)
+
+
 def test_validate_csr():
     losa = lib()
     off, idx = util.random_csr(50, 40, 3)
