@@ -35,13 +35,18 @@
 namespace losa {
 namespace {
 
-constexpr int kThreads = 384;  // 2 softmax warpgroups + 1 utility warpgroup (TMA, MMA, 2 idle warps)
+constexpr int kThreads = 384;  // 2 softmax warpgroups + 1 utility warpgroup (TMA, 2 MMA issuers, scheduler)
 constexpr int kRegsSoftmax = 216, kRegsUtility = 72, kRegsAtLaunch = 168;
 // setmaxnreg only moves registers inside the CTA's launch allocation: the increase waits until
 // the decrease has released enough, so the totals must balance or the increase never returns.
 static_assert(128 * kRegsUtility + 256 * kRegsSoftmax <= kThreads * kRegsAtLaunch,
               "register reallocation exceeds the CTA's launch allocation");
 static_assert(kThreads * kRegsAtLaunch <= 65536, "launch allocation exceeds the register file");
+// The utility warps take the LOWEST warp ids.  When several warps of a scheduler partition are
+// ready, the hardware favours the lower (older) ids; a softmax warp in an arithmetic-dense
+// stretch is ready every cycle, and with the MMA issuer behind it in that order each of the
+// issuer's instructions waited ~10x longer (measured), which put the issuer on the critical path.
+constexpr int kProducerWarp = 0, kIssuerWarp = 1, kSchedulerWarp = 3;  // issuers: warps 1 and 2
 constexpr int kTmemCols = 512;
 // Tile list ring: the scheduler warp writes one 32-bit entry per work item header, per K/V tile
 // and one end marker; every other warp reads all of them in order.
@@ -49,7 +54,6 @@ constexpr size_t kCounterBytes = 256;  // head of the workspace: the work-item c
 constexpr size_t kRowstatBytes = (size_t)kMaxPersistentCtas * 2 * 128 * sizeof(float2);
 constexpr int kTlChunks = 8;
 constexpr uint32_t kTlItem = 1u << 28, kTlEnd = 2u << 28;  // entry type in bits 31:28 (0 = tile)
-constexpr int kTlConsumers = 11;                           // producer, 2 issuers, 8 softmax warps
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;
@@ -66,10 +70,11 @@ struct Cfg {
   static constexpr int kKVBytes = kDH * kKVSlab;      // one K (or V) tile
   static constexpr bool kHasV = (MODE != kMass);
   static constexpr bool kWantMass = (MODE == kMass || MODE == kFused);
-  // Keys per S sub-tile.  With an O accumulator in TMEM there is room for two 64-column S buffers
-  // per query tile; the mass pass has no O and uses two 128-column buffers (full-rate 128-wide MMAs).
-  static constexpr int kW = (!kHasV && kC == 128) ? 128 : 64;
-  static constexpr int kSubs = kC / kW;               // sub-tiles per K/V tile
+  static constexpr int kW = kC;                       // columns of S: one K/V tile per S = Q K^T
+  // TMEM (512 columns): with an O accumulator, per query tile one S of up to 128 columns (P in
+  // place) and O; the mass pass has no O and double-buffers S instead.
+  static constexpr int kNS = kHasV ? 1 : 2;           // S buffers per query tile
+  static constexpr int kSStride = kHasV ? 128 : 256;  // TMEM columns between the tiles' S areas
   static constexpr int kRingBudget = (kHasV ? 160 : 128) * 1024;  // K + V rings
   // a V tile stays in use about one tile longer than a K tile (its products are issued one
   // sub-tile behind), so V gets the deeper ring
@@ -82,7 +87,6 @@ struct Cfg {
 
 struct Params {
   int B, H, N, nQb, nKb, nQt, nPairs, nWork;
-  int tail_subs;  // 64-key sub-tiles of the last key tile that hold valid keys
   const int32_t* offsets;
   const int32_t* kv_idx;
   void* o;
@@ -92,7 +96,7 @@ struct Params {
   float* lse;
   int* work_counter;  // zeroed before the launch; CTAs draw work items from it
   float2* rowstat;  // mass modes: [grid][2][128] final (max, 1/sum) of every row of the item
-  float2* table;  // mass modes: [grid][2][nKb * sub-tiles][128] (sum of p, reference max) per row and sub-tile
+  float2* table;  // mass modes: [grid][2][nKb][128] (sum of p, reference max) per row and key tile
   float scale_log2;
   int* status;
 };
@@ -102,13 +106,15 @@ struct Control {
   uint64_t q_full[2], q_empty[2];
   uint64_t k_full[NK], k_empty[NK];
   uint64_t v_full[NV > 0 ? NV : 1], v_empty[NV > 0 ? NV : 1];
-  uint64_t s_full[2][2], p_ready[2][2];  // per query tile and S buffer
-  uint64_t pv_done[2], o_done[2], o_free[2];  // per product / per item / O read out
+  uint64_t s_full[2][2], s_free[2][2];  // per query tile and S buffer: written by the MMAs / read out
+  uint64_t p_ready[2];                  // per query tile: P is in TMEM
+  uint64_t o_done[2], o_free[2];  // per item: all products done / O read out
   uint64_t wg_bar[2];
   uint64_t tl_full[kTlChunks], tl_empty[kTlChunks];  // tile list ring, per 32-entry chunk
   uint32_t tl[kTlChunks * 32];
   uint64_t drain;
   uint32_t tmem_base;
+  uint32_t mma_lock;  // held while a burst of MMAs is issued
   int abort_flag;
 };
 
@@ -204,27 +210,18 @@ struct TileIter {
   }
 };
 
-// Optional phase timers (diagnostic builds only, -DLOSA_PHASE_TIMERS): clock64() deltas summed
-// per phase by one thread of each role and written to the workspace pointer at the end.
-#ifdef LOSA_PHASE_TIMERS
-#define PT_DECL() long long pt_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long pt_t = clock64()
-#define PT_MARK(i)                 \
-  do {                             \
-    const long long t_ = clock64(); \
-    pt_[i] += t_ - pt_t;           \
-    pt_t = t_;                     \
-  } while (0)
-#define PT_FLUSH(role)                                                                   \
-  do {                                                                                   \
-    if ((MODE == kDense || MODE == kSparse) && p.table != nullptr && lane == 0) {                           \
-      long long* dst = reinterpret_cast<long long*>(p.table) + ((int64_t)blockIdx.x * 4 + (role)) * 8; \
-      for (int i_ = 0; i_ < 8; ++i_) dst[i_] = pt_[i_];                                  \
-    }                                                                                    \
+// Event trace (diagnostic builds only, -DLOSA_TRACE): CTA 0 records (clock, event, counter) per role.
+#ifdef LOSA_TRACE
+__device__ unsigned long long g_trace[8][4096];
+#define TR_DECL(role) unsigned long long* tr_ = g_trace[role]; int tr_n = 0; const bool tr_on = (blockIdx.x == 0 && lane == 0)
+#define TR(ev, n)                                                                           \
+  do {                                                                                      \
+    if (tr_on && tr_n < 4096)                                                               \
+      tr_[tr_n++] = ((unsigned long long)clock64() << 24) | ((unsigned long long)((n) & 0xffff) << 8) | (ev); \
   } while (0)
 #else
-#define PT_DECL() do {} while (0)
-#define PT_MARK(i) do {} while (0)
-#define PT_FLUSH(role) do {} while (0)
+#define TR_DECL(role) do {} while (0)
+#define TR(ev, n) do {} while (0)
 #endif
 
 #define LOSA_WAIT_RELAXED(bar, parity)                                   \
@@ -279,7 +276,8 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                  const __grid_constant__ CUtensorMap map_v, const Params p) {
   using C = Cfg<D, BLK, MODE>;
   using Ctl = Control<C::kNK, C::kNV>;
-  constexpr int kC = C::kC, kQBT = C::kQBT, kNB = C::kNB, kW = C::kW, kSubs = C::kSubs;
+  constexpr int kC = C::kC, kQBT = C::kQBT, kNB = C::kNB, kW = C::kW, kNS = C::kNS;
+  constexpr uint32_t kSStride = C::kSStride, kNVs = C::kNV > 0 ? C::kNV : 1;
   constexpr uint32_t kQMask = (1u << kQBT) - 1u;
 
   extern __shared__ uint8_t smem_raw[];
@@ -296,18 +294,18 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(&ctl->q_full[i], 1);
       ptx::mbar_init(&ctl->q_empty[i], 1);
-      ptx::mbar_init(&ctl->s_full[i][0], 1);
-      ptx::mbar_init(&ctl->s_full[i][1], 1);
-      ptx::mbar_init(&ctl->p_ready[i][0], 4);  // one elected arrival per softmax warp
-      ptx::mbar_init(&ctl->p_ready[i][1], 4);
-      ptx::mbar_init(&ctl->pv_done[i], 1);
+      for (int u = 0; u < 2; ++u) {
+        ptx::mbar_init(&ctl->s_full[i][u], 1);
+        ptx::mbar_init(&ctl->s_free[i][u], 4);  // one elected arrival per softmax warp
+      }
+      ptx::mbar_init(&ctl->p_ready[i], 4);  // one elected arrival per softmax warp
       ptx::mbar_init(&ctl->o_done[i], 1);
       ptx::mbar_init(&ctl->o_free[i], 128);
       ptx::mbar_init(&ctl->wg_bar[i], 128);
     }
     for (int i = 0; i < C::kNK; ++i) {
       ptx::mbar_init(&ctl->k_full[i], 1);
-      ptx::mbar_init(&ctl->k_empty[i], 2);  // both MMA issuers hand a stage back
+      ptx::mbar_init(&ctl->k_empty[i], 2);  // one arrival per query tile
     }
     for (int i = 0; i < C::kNV; ++i) {
       ptx::mbar_init(&ctl->v_full[i], 1);
@@ -315,17 +313,19 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
     for (int i = 0; i < kTlChunks; ++i) {
       ptx::mbar_init(&ctl->tl_full[i], 1);
-      ptx::mbar_init(&ctl->tl_empty[i], kTlConsumers);
+      // readers of the tile list: producer, 2 MMA issuers, 8 softmax warps
+      ptx::mbar_init(&ctl->tl_empty[i], 11);
     }
-    ptx::mbar_init(&ctl->drain, 2);  // both MMA issuers arrive on the abort path
+    ptx::mbar_init(&ctl->drain, 2);  // the MMA issuers arrive on the abort path
+    ctl->mma_lock = 0;
     ctl->abort_flag = 0;
     ptx::fence_barrier_init();
   }
-  if (warp == 9) {
+  if (warp == kIssuerWarp) {
     ptx::tmem_alloc(&ctl->tmem_base, kTmemCols);
     ptx::tmem_relinquish_alloc_permit();
   }
-  if (warp == 8 && lane == 0) {
+  if (warp == kProducerWarp && lane == 0) {
     ptx::prefetch_tensormap(&map_q);
     ptx::prefetch_tensormap(&map_k);
     if (C::kHasV) ptx::prefetch_tensormap(&map_v);
@@ -335,16 +335,15 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = ctl->tmem_base;
 
-  // The softmax warpgroups hold a whole S row per thread: the utility warpgroup (warps 8-11)
-  // gives registers up and the softmax warpgroups take them.
-  if (warp >= 8) {
+  // The softmax warpgroups hold a whole S row per thread: the utility warpgroup gives registers
+  // up and the softmax warpgroups take them.
+  if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsUtility));
-  if (warp == 8) {
+  if (warp == kProducerWarp) {
     // ------------------------------------------------------------------ TMA producer
     // (the whole warp walks the tile list; lane 0 alone issues the copies)
     {
       uint32_t nq[2] = {0, 0}, nk = 0, nv = 0, te = 0, ent;
-      PT_DECL();
       LOSA_TL_NEXT(ent);
       while ((ent >> 28) == 1) {
         const int w = (int)(ent & 0x0fffffffu);
@@ -354,9 +353,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         for (int qt = 0; qt < 2; ++qt) {
           const int T = 2 * pr + qt;
           if (T < p.nQt) {
-            PT_MARK(0);
             LOSA_WAIT_RELAXED(&ctl->q_empty[qt], (nq[qt] & 1) ^ 1);
-            PT_MARK(1);
             if (lane == 0) {
               ptx::mbar_arrive_expect_tx(&ctl->q_full[qt], C::kQBytes);
 #pragma unroll
@@ -372,9 +369,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if ((ent >> 28) != 0) break;
           const int j = (int)(ent & 0xffffu);
           const uint32_t ks = nk % C::kNK;
-          PT_MARK(0);
           LOSA_WAIT_RELAXED(&ctl->k_empty[ks], ((nk / C::kNK) & 1) ^ 1);
-          PT_MARK(2);
           if (lane == 0) {
             ptx::mbar_arrive_expect_tx(&ctl->k_full[ks], C::kKVBytes);
 #pragma unroll
@@ -384,10 +379,8 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
           ++nk;
           if (C::kHasV) {
-            const uint32_t vs = nv % (C::kNV > 0 ? C::kNV : 1);
-            PT_MARK(0);
-            LOSA_WAIT_RELAXED(&ctl->v_empty[vs], ((nv / (C::kNV > 0 ? C::kNV : 1)) & 1) ^ 1);
-            PT_MARK(3);
+            const uint32_t vs = nv % kNVs;
+            LOSA_WAIT_RELAXED(&ctl->v_empty[vs], ((nv / kNVs) & 1) ^ 1);
             if (lane == 0) {
               ptx::mbar_arrive_expect_tx(&ctl->v_full[vs], C::kKVBytes);
 #pragma unroll
@@ -399,133 +392,123 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
         }
       }
-      PT_MARK(0);
-      PT_FLUSH(2);
     }
-  } else if (warp == 9 || warp == 10) {
+  } else if (warp == kIssuerWarp || warp == kIssuerWarp + 1) {
     // ------------------------------------------------------------------ MMA issuers
-    // One issuing warp per query tile (warp 9: tile 0, warp 10: tile 1), so that a wait in one
-    // tile's chain never delays the other tile's MMAs.  Each walks every tile of the item in
-    // order (whole warp, for the shared index window); lane 0 alone issues MMAs and commits.
-    //
-    // A key tile is consumed as 64-key sub-tiles, and the S accumulator of a query tile is
-    // double-buffered (2 x 64 TMEM columns): S(n+1) = Q K(n+1)^T is issued before O += P(n) V(n),
-    // so the tensor pipe works on sub-tile n+1 and n-1 while the softmax warpgroup is busy
-    // with sub-tile n.  Up to two P V products are pending at any time.
+    // One warp per query tile (lane 0 issues).  Per key tile that the query tile lists it runs
+    //   S = Q K^T  ->  (softmax warps turn S into P, in place)  ->  O += P V
+    // and only then S of the next key tile, because P lives in the columns of S.  That chain is
+    // serial per query tile; the two query tiles run it half a period apart, so that one tile's
+    // MMAs execute while the other tile's softmax runs and the two warpgroups do not compete
+    // for the exponential unit.  The half-period offset is kept by a lock: a burst (O += P V
+    // of one key tile, then S of the next) is issued whole, never interleaved with the other
+    // tile's burst - interleaved bursts finish together and lock the tiles in step.
+    // The mass pass has no P and no O: there S is double-buffered and handed back by the
+    // softmax warps as soon as it is read.
     {
-      const int qt = warp - 9;
+      const int qt = warp - kIssuerWarp;
       const bool leader = (lane == 0);
-      const uint32_t q_base = ptx::smem_u32(sQ), k_base = ptx::smem_u32(sK),
-                     v_base = ptx::smem_u32(sV);
-      uint32_t nq = 0, nt = 0, nsub = 0, npv = 0, nof = 0, te = 0, ent;
-      // nt: tiles walked, nsub: S sub-tiles issued, npv: P V products issued (kernel lifetime)
-      PT_DECL();
-
+      uint32_t nq = 0, nt = 0, nsub = 0, nof = 0, te = 0, ent;
+      TR_DECL(2 + qt);
       constexpr uint32_t kDescHi = ptx::smem_desc_hi_sw128(1024);
-      const uint32_t q_lo = ptx::smem_desc_lo(q_base, 16) + qt * (C::kQBytes >> 4);
-      const uint32_t k_lo = ptx::smem_desc_lo(k_base, 16);
-      const uint32_t v_lo = ptx::smem_desc_lo(v_base, C::kKVSlab);
-      const uint32_t tS = tmem_base + qt * 2 * kW, tO = tmem_base + 256 + qt * 128;
-      constexpr uint32_t kNVs = C::kNV > 0 ? C::kNV : 1;
-
-      // S[buf] = Q K(stage ks, sub-tile h)^T
-      auto issue_qk = [&](uint32_t ks, int h, uint32_t buf) {
-        if (!leader) return;
-        const uint32_t b0 = k_lo + ks * (C::kKVBytes >> 4) + ((h * kW * 128) >> 4);
+      const uint32_t k_lo = ptx::smem_desc_lo(ptx::smem_u32(sK), 16);
+      const uint32_t v_lo = ptx::smem_desc_lo(ptx::smem_u32(sV), C::kKVSlab);
+      const uint32_t tS = tmem_base + qt * kSStride;
+      const uint32_t tO = tmem_base + 256 + qt * 128;
+      // every descriptor is built before the waits, so that the MMAs issue back to back
+      uint64_t qd[D / 16];
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t a_off = ((kk >> 2) * C::kQSlab + (kk & 3) * 32) >> 4;
-          const uint32_t b_off = ((kk >> 2) * C::kKVSlab + (kk & 3) * 32) >> 4;
-          ptx::mma_ss_lohi(tS + buf * kW, q_lo + a_off, b0 + b_off, kDescHi, C::kIdescQK,
-                           kk > 0 ? 1u : 0u);
-        }
-      };
-      // O (+)= P[buf] V(stage vs, keys 64 h .. 64 h + 63)
-      auto issue_pv = [&](uint32_t vs, int h, uint32_t buf, bool accumulate) {
-        if (!leader) return;
-        const uint32_t b0 = v_lo + vs * (C::kKVBytes >> 4) + ((h * 64 * 128) >> 4);
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk)
-          ptx::mma_ts_lohi(tO, tS + buf * 64 + kk * 8, b0 + kk * (2048 >> 4), kDescHi,
-                           C::kIdescPV, (accumulate || kk > 0) ? 1u : 0u);
-      };
-
-      // pending P V products, oldest first: V stage, its phase, sub-tile, last-of-tile flag
-      // (kept in scalars: slot 0 is the oldest, slot 1 the newest)
-      uint32_t pd_vs0 = 0, pd_ph0 = 0, pd_tile0 = 0, pd_vs1 = 0, pd_ph1 = 0, pd_tile1 = 0;
-      int pd_h0 = 0, pd_h1 = 0;
-      bool pd_last0 = false, pd_last1 = false;
-      int npend = 0;
-      uint32_t pv_item = 0;
-
-#define LOSA_POP_PV()                                                              \
-  do {                                                                             \
-    PT_MARK(0);                                                                    \
-    if (C::kHasV) LOSA_WAIT(&ctl->v_full[pd_vs0], pd_ph0);                     \
-    PT_MARK(1);                                                                    \
-    LOSA_WAIT(&ctl->p_ready[qt][npv & 1], (npv >> 1) & 1);                         \
-    PT_MARK(2);                                                                    \
-    if (C::kHasV) {                                                                \
-      if (pv_item == 0 && nof > 0) LOSA_WAIT(&ctl->o_free[qt], (nof - 1) & 1);     \
-      ptx::tc_fence_after_sync();                                                  \
-      issue_pv(pd_vs0, pd_h0, npv & 1, pv_item > 0);                           \
-      PT_MARK(4);                                                                  \
-      if (leader) {                                                                \
-        ptx::mma_commit(&ctl->pv_done[qt]);                                        \
-        if (pd_last0) ptx::mma_commit(&ctl->v_empty[pd_vs0]);                  \
-      }                                                                            \
-      ++pv_item;                                                                   \
-    }                                                                              \
-    ++npv;                                                                         \
-    pd_vs0 = pd_vs1; pd_ph0 = pd_ph1; pd_h0 = pd_h1;                               \
-    pd_last0 = pd_last1; pd_tile0 = pd_tile1;                                      \
-    --npend;                                                                       \
-    PT_MARK(6);                                                                    \
-  } while (0)
+      for (int kk = 0; kk < D / 16; ++kk)
+        qd[kk] = ptx::desc64(ptx::smem_desc_lo(ptx::smem_u32(sQ), 16) + qt * (C::kQBytes >> 4) +
+                                 (((kk >> 2) * C::kQSlab + (kk & 3) * 32) >> 4),
+                             kDescHi);
 
       LOSA_TL_NEXT(ent);
       while ((ent >> 28) == 1) {
-        bool q_ready = false;
-        pv_item = 0;
+        bool q_ready = false, pend = false;
+        uint32_t pend_vs = 0, pend_vph = 0, pv_item = 0;
         for (;;) {
           LOSA_TL_NEXT(ent);
-          if ((ent >> 28) != 0) break;
-          const int j = (int)(ent & 0xffffu);
+          const bool more = (ent >> 28) == 0;
           const uint32_t memb = (ent >> 16) & 0xfu;
           const uint32_t ks = nt % C::kNK, kph = (nt / C::kNK) & 1;
           const uint32_t vs = nt % kNVs, vph = (nt / kNVs) & 1;
-          const bool member = ((memb >> (qt * kQBT)) & kQMask) != 0;
-          const int subs = (j == p.nKb - 1) ? p.tail_subs : kSubs;
-          PT_MARK(0);
-          LOSA_WAIT(&ctl->k_full[ks], kph);
-          PT_MARK(1);
-          // V stages go back to the producer in tile order, and the producer refills this
-          // tile's stage only after its previous user was handed back: finish the pending
-          // products of any tile that used this V stage before.
-          while (C::kHasV && npend > 0 && pd_tile0 + kNVs <= nt) LOSA_POP_PV();
+          const bool member = more && ((memb >> (qt * kQBT)) & kQMask) != 0;
+          const uint32_t buf = nsub % kNS;
+          uint64_t kd[D / 16], vd[kW / 16];
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk)
+            kd[kk] = ptx::desc64(k_lo + ks * (C::kKVBytes >> 4) +
+                                     (((kk >> 2) * C::kKVSlab + (kk & 3) * 32) >> 4),
+                                 kDescHi);
+#pragma unroll
+          for (int kk = 0; kk < kW / 16; ++kk)
+            vd[kk] = ptx::desc64(v_lo + pend_vs * (C::kKVBytes >> 4) + kk * (2048 >> 4), kDescHi);
+          // operands first, the softmax hand-over last: it is the wait that ends latest
+          if (more) LOSA_WAIT(&ctl->k_full[ks], kph);
           if (member) {
             if (!q_ready) {
               LOSA_WAIT(&ctl->q_full[qt], nq & 1);
               ++nq;
               q_ready = true;
             }
-            for (int h = 0; h < subs; ++h) {
-              if (npend == 2) LOSA_POP_PV();  // frees the S buffer this sub-tile will use
-              ptx::tc_fence_after_sync();
-              issue_qk(ks, h, nsub & 1);
-              PT_MARK(5);
-              if (leader) ptx::mma_commit(&ctl->s_full[qt][nsub & 1]);
-              if (npend == 0) {
-                pd_vs0 = vs; pd_ph0 = vph; pd_h0 = h; pd_tile0 = nt; pd_last0 = (h == subs - 1);
-              } else {
-                pd_vs1 = vs; pd_ph1 = vph; pd_h1 = h; pd_tile1 = nt; pd_last1 = (h == subs - 1);
+            // mass pass: the S buffer is free once the softmax warps have read its last content
+            if (!C::kHasV && nsub >= (uint32_t)kNS)
+              LOSA_WAIT(&ctl->s_free[qt][buf], ((nsub / kNS) - 1) & 1);
+          }
+          if (C::kHasV && pend) {
+            LOSA_WAIT(&ctl->v_full[pend_vs], pend_vph);
+            if (pv_item == 0 && nof > 0) LOSA_WAIT(&ctl->o_free[qt], (nof - 1) & 1);
+            TR(1, nsub);
+            LOSA_WAIT(&ctl->p_ready[qt], (nsub - 1) & 1);
+            TR(2, nsub);
+          }
+          if ((C::kHasV && pend) || member) {
+            // ---- one burst, under the lock
+            if (leader) {
+              uint32_t it = 0;
+              while (atomicCAS(&ctl->mma_lock, 0u, 1u) != 0u) {
+                if (++it > (1u << 22) || ctl->abort_flag) break;  // bounded; the wait below reports it
+                __nanosleep(32);
               }
-              ++npend;
-              ++nsub;
-              PT_MARK(6);
             }
-            if (leader) ptx::mma_commit(&ctl->k_empty[ks]);
+            __syncwarp();
+            ptx::tc_fence_after_sync();
+            if (leader) {
+              if (C::kHasV && pend) {
+                // O += P V for the previous key tile of this query tile
+                ptx::mma_ts_d(tO, tS, vd[0], C::kIdescPV, pv_item > 0 ? 1u : 0u);
+#pragma unroll
+                for (int kk = 1; kk < kW / 16; ++kk)
+                  ptx::mma_ts_d(tO, tS + kk * 8, vd[kk], C::kIdescPV, 1u);
+                ptx::mma_commit(&ctl->v_empty[pend_vs]);
+              }
+              if (member) {
+                ptx::mma_ss_d(tS + buf * 128, qd[0], kd[0], C::kIdescQK, 0u);
+#pragma unroll
+                for (int kk = 1; kk < D / 16; ++kk)
+                  ptx::mma_ss_d(tS + buf * 128, qd[kk], kd[kk], C::kIdescQK, 1u);
+                // completes after every MMA issued so far, the tile's last O += P V included
+                ptx::mma_commit(&ctl->s_full[qt][buf]);
+                ptx::mma_commit(&ctl->k_empty[ks]);
+              }
+              __threadfence_block();
+              atomicExch(&ctl->mma_lock, 0u);
+            }
+            TR(3, nsub);
+          }
+          if (C::kHasV && pend) {
+            ++pv_item;
+            pend = false;
+          }
+          if (!more) break;
+          if (member) {
+            ++nsub;
+            pend = C::kHasV;
+            pend_vs = vs;
+            pend_vph = vph;
           } else {
+            // the copies must have landed before a stage is handed back
             if (leader) ptx::mbar_arrive(&ctl->k_empty[ks]);
             if (C::kHasV) {
               LOSA_WAIT(&ctl->v_full[vs], vph);
@@ -534,19 +517,15 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
           ++nt;
         }
-        while (npend > 0) LOSA_POP_PV();
-        if (q_ready && leader) ptx::mma_commit(&ctl->q_empty[qt]);
-        if (pv_item > 0) {
+        if (C::kHasV && pv_item > 0) {
           if (leader) ptx::mma_commit(&ctl->o_done[qt]);  // every product of the item is done
           ++nof;
         }
+        if (q_ready && leader) ptx::mma_commit(&ctl->q_empty[qt]);
       }
-#undef LOSA_POP_PV
-      PT_MARK(0);
-      if (qt == 0) PT_FLUSH(3);
     }
-  } else {
-    // ------------------------------------------------------------------ scheduler (warp 11)
+  } else if (warp == kSchedulerWarp) {
+    // ------------------------------------------------------------------ scheduler
     // Walks the block-index lists of this CTA's work items and publishes, per item, a header
     // and the ascending merge of its tiles; nobody else touches the CSR.
     uint32_t te = 0;
@@ -574,17 +553,17 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   } else {
     // ------------------------------------------------------------------ softmax warpgroups
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-    const int qt = warp >> 2, wl = warp & 3;
+    const int qt = (warp >> 2) - 1, wl = warp & 3;  // TMEM lanes 32 * (warp % 4) .. + 31
     const int row = wl * 32 + lane;
     const uint32_t lane_base = (uint32_t)(wl * 32) << 16;
-    const uint32_t tS = tmem_base + lane_base + qt * 2 * kW;
+    const uint32_t tS = tmem_base + lane_base + qt * kSStride;  // P overwrites its first kW/2 columns
     const uint32_t tO = tmem_base + lane_base + 256 + qt * 128;
     const int sub = (BLK == 64) ? (wl >> 1) : 0;
     const int my_bit = qt * kQBT + sub;
     const int tail = p.N - (p.nKb - 1) * kC;  // valid keys of the last K/V tile
-    uint32_t nsub = 0, nwg = 0, nod = 0;      // nsub: sub-tiles of this query tile so far
+    uint32_t nsub = 0, nwg = 0, nod = 0;      // nsub: key tiles of this query tile so far
     uint32_t te = 0, ent;
-    PT_DECL();
+    TR_DECL((wl == 0) ? qt : 7);
 
     LOSA_TL_NEXT(ent);
     while ((ent >> 28) == 1) {
@@ -597,7 +576,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       uint32_t pv_item = 0;
       float2* tab = nullptr;
       if (C::kWantMass)
-        tab = p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * kSubs * 128 + row;
+        tab = p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * 128 + row;
       for (;;) {
         LOSA_TL_NEXT(ent);
         if ((ent >> 28) != 0) break;
@@ -605,110 +584,112 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint32_t memb = (ent >> 16) & 0xfu;
         if (((memb >> (qt * kQBT)) & kQMask) == 0) continue;
         const bool mine = (memb >> my_bit) & 1u;
-        const int subs = (j == p.nKb - 1) ? p.tail_subs : kSubs;
-        for (int hs = 0; hs < subs; ++hs) {
-          const uint32_t buf = nsub & 1, ph = (nsub >> 1) & 1;
-          const uint32_t tSb = tS + buf * kW;
-          PT_MARK(0);
-          LOSA_WAIT(&ctl->s_full[qt][buf], ph);
-          PT_MARK(1);
-          ptx::tc_fence_after_sync();
-          if (mine) {
-            uint32_t sr[kW];
+        const uint32_t buf = nsub % kNS;
+        const uint32_t tSb = tS + buf * 128;
+        // S of this key tile is complete, and so is every earlier product into O
+        TR(1, nsub);
+        LOSA_WAIT(&ctl->s_full[qt][buf], (nsub / kNS) & 1);
+        TR(2, nsub);
+        ptx::tc_fence_after_sync();
+        uint32_t sr[kW];
+        if (mine) {
 #pragma unroll
-            for (int c0 = 0; c0 < kW; c0 += 32) ptx::tmem_ld32(tSb + c0, &sr[c0]);
-            ptx::tmem_wait_ld();
-            PT_MARK(2);
-            if (j == p.nKb - 1) {
-              const int valid = tail - hs * kW;  // keys >= N do not exist
-              if (valid < kW) {
-#pragma unroll
-                for (int c = 0; c < kW; ++c)
-                  if (c >= valid) sr[c] = 0xff800000u;
-              }
-            }
-            float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
-            float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
-#pragma unroll
-            for (int c = 4; c + 8 <= kW; c += 8) {
-              mx0 = ptx::max3(mx0, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
-              mx1 = ptx::max3(mx1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
-              mx2 = ptx::max3(mx2, __uint_as_float(sr[c + 4]), __uint_as_float(sr[c + 5]));
-              mx3 = ptx::max3(mx3, __uint_as_float(sr[c + 6]), __uint_as_float(sr[c + 7]));
-            }
-            mx0 = ptx::max3(mx0, __uint_as_float(sr[kW - 4]), __uint_as_float(sr[kW - 3]));
-            mx1 = ptx::max3(mx1, __uint_as_float(sr[kW - 2]), __uint_as_float(sr[kW - 1]));
-            const float m_new =
-                fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
-            const bool need = m_new > m_ref + kRescaleThreshold;
-            if (__any_sync(0xffffffffu, need)) {
-              const float alpha = need ? ptx::ex2_approx(m_ref - m_new) : 1.f;
-              if (need) m_ref = m_new;
-              l *= alpha;
-              if (C::kHasV && pv_item > 0) {
-                // O may only be touched once the previous product of this query tile is done
-                LOSA_WAIT(&ctl->pv_done[qt], (nsub - 1) & 1);
-                ptx::tc_fence_after_sync();
-                const float2 a2 = make_float2(alpha, alpha);
-#pragma unroll
-                for (int c0 = 0; c0 < D; c0 += 32) {
-                  uint32_t r[32];
-                  ptx::tmem_ld32(tO + c0, r);
-                  ptx::tmem_wait_ld();
-#pragma unroll
-                  for (int c = 0; c < 32; c += 2) {
-                    const float2 v = ptx::mul2(
-                        make_float2(__uint_as_float(r[c]), __uint_as_float(r[c + 1])), a2);
-                    r[c] = __float_as_uint(v.x);
-                    r[c + 1] = __float_as_uint(v.y);
-                  }
-                  ptx::tmem_st32(tO + c0, r);
-                }
-              }
-            }
-            // p = 2^(s * scale_log2 - m_ref), two columns per instruction; the bf16 pairs
-            // overwrite the low half of the register array
-            PT_MARK(3);
-            const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
-            const float2 nm2 = make_float2(-m_ref, -m_ref);
-            float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int c = 0; c < kW; c += 4) {
-              float2 x0 = ptx::fma2(
-                  make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2);
-              float2 x1 = ptx::fma2(
-                  make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, nm2);
-              x0.x = ptx::ex2_approx(x0.x);
-              x0.y = ptx::ex2_approx(x0.y);
-              x1.x = ptx::ex2_approx(x1.x);
-              x1.y = ptx::ex2_approx(x1.y);
-              acc0 = ptx::add2(acc0, x0);
-              acc1 = ptx::add2(acc1, x1);
-              sr[c >> 1] = ptx::pack_bf16x2(x0.x, x0.y);
-              sr[(c >> 1) + 1] = ptx::pack_bf16x2(x1.x, x1.y);
-            }
-            PT_MARK(4);
-            const float tsum = (acc0.x + acc0.y) + (acc1.x + acc1.y);
-            l += tsum;
-            if (C::kHasV) ptx::tmem_st32(tSb, sr);
-            if (C::kWantMass) tab[((int64_t)j * kSubs + hs) * 128] = make_float2(tsum, m_ref);
-          } else if (C::kHasV) {
-            // this half of the 128-row tile does not list the key block: P = 0
-            uint32_t z[32];
-#pragma unroll
-            for (int c = 0; c < 32; ++c) z[c] = 0u;
-            ptx::tmem_st32(tSb, z);
-          }
-          if (C::kHasV) {
-            ptx::tmem_wait_st();
-            ++pv_item;
-          }
+          for (int c0 = 0; c0 < kW; c0 += 32) ptx::tmem_ld32(tSb + c0, &sr[c0]);
+          ptx::tmem_wait_ld();
+        }
+        TR(3, nsub);
+        if (!C::kHasV) {
+          // mass pass: S is in registers, hand the buffer back
           ptx::tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(&ctl->p_ready[qt][buf]);
-          ++nsub;
-          PT_MARK(5);
+          if (lane == 0) ptx::mbar_arrive(&ctl->s_free[qt][buf]);
         }
+        if (mine) {
+          if (j == p.nKb - 1 && tail < kW) {  // keys >= N do not exist
+#pragma unroll
+            for (int c = 0; c < kW; ++c)
+              if (c >= tail) sr[c] = 0xff800000u;
+          }
+          float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
+          float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
+#pragma unroll
+          for (int c = 4; c + 8 <= kW; c += 8) {
+            mx0 = ptx::max3(mx0, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
+            mx1 = ptx::max3(mx1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
+            mx2 = ptx::max3(mx2, __uint_as_float(sr[c + 4]), __uint_as_float(sr[c + 5]));
+            mx3 = ptx::max3(mx3, __uint_as_float(sr[c + 6]), __uint_as_float(sr[c + 7]));
+          }
+          mx0 = ptx::max3(mx0, __uint_as_float(sr[kW - 4]), __uint_as_float(sr[kW - 3]));
+          mx1 = ptx::max3(mx1, __uint_as_float(sr[kW - 2]), __uint_as_float(sr[kW - 1]));
+          const float m_new =
+              fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
+          const bool need = m_new > m_ref + kRescaleThreshold;
+          TR(4, nsub);
+          if (__any_sync(0xffffffffu, need)) {
+            const float alpha = need ? ptx::ex2_approx(m_ref - m_new) : 1.f;
+            if (need) m_ref = m_new;
+            l *= alpha;
+            if (C::kHasV && pv_item > 0) {
+              const float2 a2 = make_float2(alpha, alpha);
+#pragma unroll
+              for (int c0 = 0; c0 < D; c0 += 32) {
+                uint32_t r[32];
+                ptx::tmem_ld32(tO + c0, r);
+                ptx::tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 32; c += 2) {
+                  const float2 v = ptx::mul2(
+                      make_float2(__uint_as_float(r[c]), __uint_as_float(r[c + 1])), a2);
+                  r[c] = __float_as_uint(v.x);
+                  r[c + 1] = __float_as_uint(v.y);
+                }
+                ptx::tmem_st32(tO + c0, r);
+              }
+            }
+          }
+          // p = 2^(s * scale_log2 - m_ref), two columns per instruction; the bf16 pairs
+          // overwrite the low half of the register array
+          TR(5, nsub);
+          const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+          const float2 nm2 = make_float2(-m_ref, -m_ref);
+          float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+#pragma unroll
+          for (int c = 0; c < kW; c += 4) {
+            float2 x0 = ptx::fma2(
+                make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2);
+            float2 x1 = ptx::fma2(
+                make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, nm2);
+            x0.x = ptx::ex2_approx(x0.x);
+            x0.y = ptx::ex2_approx(x0.y);
+            x1.x = ptx::ex2_approx(x1.x);
+            x1.y = ptx::ex2_approx(x1.y);
+            acc0 = ptx::add2(acc0, x0);
+            acc1 = ptx::add2(acc1, x1);
+            sr[c >> 1] = ptx::pack_bf16x2(x0.x, x0.y);
+            sr[(c >> 1) + 1] = ptx::pack_bf16x2(x1.x, x1.y);
+            if (C::kHasV && (c & 63) == 60) ptx::tmem_st32(tSb + (c >> 6) * 32, &sr[(c >> 6) * 32]);
+          }
+          TR(6, nsub);
+          const float tsum = (acc0.x + acc0.y) + (acc1.x + acc1.y);
+          l += tsum;
+          if (C::kWantMass) tab[(int64_t)j * 128] = make_float2(tsum, m_ref);
+        } else if (C::kHasV) {
+          // this half of the 128-row tile does not list the key block: P = 0
+          uint32_t z[32];
+#pragma unroll
+          for (int c = 0; c < 32; ++c) z[c] = 0u;
+#pragma unroll
+          for (int c0 = 0; c0 < kW / 2; c0 += 32) ptx::tmem_st32(tSb + c0, z);
+        }
+        if (C::kHasV) {
+          ptx::tmem_wait_st();
+          ++pv_item;
+          ptx::tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&ctl->p_ready[qt]);
+          TR(7, nsub);
+        }
+        ++nsub;
       }
 
       if (C::kHasV) {
@@ -718,7 +699,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const float inv = (l > 0.f) ? 1.f / l : 0.f;
           const int64_t off = (int64_t)b * p.sb + (int64_t)h * p.sh + (int64_t)grow * p.sn;
           if (pv_item > 0) {
-            // o_done advances once per item, so its parity is unambiguous here (pv_done may be
+            // o_done advances once per item, so its parity is unambiguous here (a product's own barrier may be
             // one, two or three phases from this warp's last look at it)
             LOSA_WAIT(&ctl->o_done[qt], nod & 1);
             ++nod;
@@ -777,24 +758,21 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         ++nwg;
         if (T < p.nQt) {
           const float2* tb =
-              p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * kSubs * 128;
+              p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * 128;
           float2 st[4];  // this lane's four rows
 #pragma unroll
           for (int rr = 0; rr < 4; ++rr) st[rr] = rs[rr * 32 + lane];
           for (int u = wl; u < p.nKb; u += 4) {
-            const int subs = (u == p.nKb - 1) ? p.tail_subs : kSubs;
             float acc[kQBT];
 #pragma unroll
             for (int q = 0; q < kQBT; ++q) acc[q] = 0.f;
-            for (int hs = 0; hs < subs; ++hs) {
 #pragma unroll
-              for (int rr = 0; rr < 4; ++rr) {
-                const int r = rr * 32 + lane;
-                const float2 tv = tb[((int64_t)u * kSubs + hs) * 128 + r];
-                const float wgt =
-                    (st[rr].y > 0.f) ? tv.x * ptx::ex2_approx(tv.y - st[rr].x) * st[rr].y : 0.f;
-                acc[(rr * 32) / BLK] += wgt;
-              }
+            for (int rr = 0; rr < 4; ++rr) {
+              const int r = rr * 32 + lane;
+              const float2 tv = tb[(int64_t)u * 128 + r];
+              const float wgt =
+                  (st[rr].y > 0.f) ? tv.x * ptx::ex2_approx(tv.y - st[rr].x) * st[rr].y : 0.f;
+              acc[(rr * 32) / BLK] += wgt;
             }
 #pragma unroll
             for (int q = 0; q < kQBT; ++q) {
@@ -813,29 +791,27 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         LOSA_WAIT(&ctl->wg_bar[qt], nwg & 1);
         ++nwg;
       }
-      PT_MARK(6);  // epilogue of the item
     }
-    if (wl == 0) PT_FLUSH(qt);
   }
 
 teardown:
   if (ctl->abort_flag) {
     // Abort path: give MMAs and bulk copies still in flight a bounded time to land before
     // shared memory and TMEM are released.
-    if ((warp == 9 || warp == 10) && lane == 0) {
+    if ((warp == kIssuerWarp || warp == kIssuerWarp + 1) && lane == 0) {
       ptx::mma_commit(&ctl->drain);
       for (uint32_t it = 0; it < (1u << 16); ++it) {
         if (ptx::mbar_try_wait(&ctl->drain, 0)) break;
         __nanosleep(128);
       }
     }
-    if (warp == 8 && lane == 0) {
+    if (warp == kProducerWarp && lane == 0) {
       for (uint32_t it = 0; it < (1u << 10); ++it) __nanosleep(1024);
     }
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
-  if (warp == 9) {
+  if (warp == kIssuerWarp) {
     ptx::tc_fence_after_sync();
     ptx::tmem_dealloc(tmem_base, kTmemCols);
   }
@@ -943,13 +919,17 @@ int dispatch(const Geometry& g, const void* q, const void* k, const void* v, con
 
 }  // namespace
 
+#ifdef LOSA_TRACE
+extern "C" int losa_debug_trace(void* host, size_t bytes) {
+  return (int)cudaMemcpyFromSymbol(host, g_trace, bytes < sizeof(g_trace) ? bytes : sizeof(g_trace));
+}
+#endif
+
 size_t attn_workspace_bytes(AttnMode mode, const Geometry& g) {
   if (mode == kDense || mode == kSparse) return kCounterBytes;
-  // counter, per-CTA row statistics, per-CTA table of one entry per row and sub-tile; the mass
-  // pass has one sub-tile per key tile, the fused pass C / 64
-  const size_t subs = (mode == kMass) ? 1 : (size_t)g.C / 64;
+  // counter, per-CTA row statistics, per-CTA table of one entry per row and key tile
   return kCounterBytes + kRowstatBytes +
-         (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * subs * 128 * sizeof(float2);
+         (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2);
 }
 
 int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, const void* v,
@@ -964,8 +944,6 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
   prm.nQt = g.nQt;
   prm.nPairs = g.nPairs;
   prm.nWork = g.B * g.H * g.nPairs;
-  const int sub_w = (mode == kMass && g.C == 128) ? 128 : 64;  // Cfg::kW
-  prm.tail_subs = (g.N - (g.nKb - 1) * g.C + sub_w - 1) / sub_w;
   prm.offsets = offsets;
   prm.kv_idx = kv_idx;
   prm.o = o;
