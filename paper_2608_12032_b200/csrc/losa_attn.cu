@@ -2,13 +2,14 @@
 // frozen CSR pattern (Eq. 4) and the exact block-mass pass (Eq. 1), as ONE warp-specialised
 // persistent kernel template.
 //
-// CTA = 12 warps.  Warps 0-3 and 4-7 are two softmax warpgroups, each owning one 128-row
-// query tile (thread = query row = TMEM lane); they take 216 registers per thread from the
-// third warpgroup (setmaxnreg), whose warps 10-11 idle.  Warp 8 (one elected thread) is the TMA
-// producer: it streams the query tiles and the K / V tiles named by the block indices into
-// 128B-swizzled shared-memory rings.  Warp 9 (one elected thread) issues the tcgen05 MMAs:
-// S = Q K^T from shared memory into TMEM, O += P V with P read from TMEM (bf16, aliasing S)
-// and V from shared memory as the MN-major operand.
+// CTA = 12 warps.  Warps 0-3 are utility warps: warp 0 (one elected thread) is the TMA producer,
+// which streams the query tiles and the K / V tiles named by the block indices into
+// 128B-swizzled shared-memory rings; warps 1 and 2 (one elected thread each) issue the tcgen05
+// MMAs of query tile 0 and 1: S = Q K^T from shared memory into TMEM, O += P V with P read from
+// TMEM (bf16, written over S) and V from shared memory as the MN-major operand; warp 3 walks
+// the block-index lists and publishes the tile list every other warp follows.  Warps 4-7 and
+// 8-11 are two softmax warpgroups, each owning one 128-row query tile (thread = query row =
+// TMEM lane); they take their registers from the utility warpgroup (setmaxnreg).
 //
 // A work item is a pair of consecutive query tiles of one (batch, head).  The key blocks the
 // pair visits are the ascending merge of the tiles' index lists (one list per query block;
@@ -16,11 +17,14 @@
 // MMAs are issued only for the query tiles that list it.  Query-block rows that do not list
 // a tile of their 128-row group get P = 0 for it.
 //
-// The MMA thread runs one tile ahead on S: after O_t += P V(u) it issues S_t = Q_t K(u+1)^T
-// for the same tile t, then turns to the other tile, so each warpgroup's softmax overlaps
-// the other tile's MMAs.  Running maxima are updated lazily: O and the row sum are rescaled
-// only when the maximum grew by more than 2^8, which keeps the correction off the common
-// path without losing accuracy (the stale reference bounds p by 2^8).
+// One S = Q K^T covers a whole key tile (for 128-key tiles, 128-wide MMAs: an MMA costs its
+// issuing thread ~70 cycles whatever its width, so wide MMAs are what keeps the issuer off the
+// critical path).  TMEM then holds exactly S and O of both query tiles, P overwrites S, and
+// per query tile the steps S -> softmax -> O += P V -> next S form a serial chain.  The two
+// tiles run that chain half a period apart: one tile's MMAs execute while the other tile's
+// softmax runs.  Running maxima are updated lazily: O and the row sum are rescaled only when
+// the maximum grew by more than 2^8, which keeps the correction off the common path without
+// losing accuracy (the stale reference bounds p by 2^8).
 //
 // Every wait is bounded; a wait that expires raises the CTA's abort flag, records
 // LOSA_ERR_TIMEOUT, and all roles leave through the common teardown that frees TMEM.
@@ -468,7 +472,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             if (leader) {
               uint32_t it = 0;
               while (atomicCAS(&ctl->mma_lock, 0u, 1u) != 0u) {
-                if (++it > (1u << 22) || ctl->abort_flag) break;  // bounded; the wait below reports it
+                if (++it > (1u << 22) || ctl->abort_flag) break;  // bounded; a later wait reports it
                 __nanosleep(32);
               }
             }
@@ -481,7 +485,6 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
                 for (int kk = 1; kk < kW / 16; ++kk)
                   ptx::mma_ts_d(tO, tS + kk * 8, vd[kk], C::kIdescPV, 1u);
-                ptx::mma_commit(&ctl->v_empty[pend_vs]);
               }
               if (member) {
                 ptx::mma_ss_d(tS + buf * 128, qd[0], kd[0], C::kIdescQK, 0u);
@@ -490,10 +493,12 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                   ptx::mma_ss_d(tS + buf * 128, qd[kk], kd[kk], C::kIdescQK, 1u);
                 // completes after every MMA issued so far, the tile's last O += P V included
                 ptx::mma_commit(&ctl->s_full[qt][buf]);
-                ptx::mma_commit(&ctl->k_empty[ks]);
               }
-              __threadfence_block();
-              atomicExch(&ctl->mma_lock, 0u);
+              // the lock orders the issue of bursts, not data: a plain store releases it
+              *reinterpret_cast<volatile uint32_t*>(&ctl->mma_lock) = 0u;
+              // stages go back when the MMAs that read them have completed
+              if (C::kHasV && pend) ptx::mma_commit(&ctl->v_empty[pend_vs]);
+              if (member) ptx::mma_commit(&ctl->k_empty[ks]);
             }
             TR(3, nsub);
           }
