@@ -166,9 +166,12 @@ int losa_select_noalloc(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const fl
  * The CSR must satisfy losa_validate_csr(); a block index outside [0, nKb) is skipped and
  * reported as LOSA_ERR_BAD_INDEX, never dereferenced.
  *   q, k, v  bf16 [B,H,N,D];  o  [B,H,N,D] with the same strides, bf16 or f32 (o_dtype)
- *   ws       >= losa_workspace_bytes(LOSA_OP_SPARSE_ATTN, p) bytes (a few hundred: the
- *            counter the persistent CTAs draw work items from); not shared between calls
- *            that may run concurrently                                                    */
+ *   ws       >= losa_workspace_bytes(LOSA_OP_SPARSE_ATTN, p) bytes (about 21 MB at D = 128:
+ *            the counter the persistent CTAs draw work items from, and the partial results
+ *            of the last work items, which are processed in parts and merged by a second
+ *            kernel on the same stream); not shared between calls that may run
+ *            concurrently; contents undefined afterwards.  The result does not depend on
+ *            timing: the same call on the same GPU gives the same bits.                   */
 int losa_sparse_attn(const losa_problem_t* p, const void* q, const void* k, const void* v,
                      const int32_t* offsets, const int32_t* kv_idx, void* o, int o_dtype,
                      void* ws, size_t ws_bytes, void* cuda_stream);

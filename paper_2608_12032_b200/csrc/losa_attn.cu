@@ -56,8 +56,13 @@ constexpr int kTmemCols = 512;
 // and one end marker; every other warp reads all of them in order.
 constexpr size_t kCounterBytes = 256;  // head of the workspace: the work-item counter
 constexpr size_t kRowstatBytes = (size_t)kMaxPersistentCtas * 2 * 128 * sizeof(float2);
+constexpr size_t kPartMlBytes = kRowstatBytes;  // same shape: [slot][2][128] float2
 constexpr int kTlChunks = 8;
 constexpr uint32_t kTlItem = 1u << 28, kTlEnd = 2u << 28;  // entry type in bits 31:28 (0 = tile)
+// An item header carries the work item in bits 23:0 and, for a unit that covers only part of the
+// item's key range, the part index in bits 26:24 and a flag in bit 27.
+constexpr uint32_t kTlItemMask = 0x00ffffffu, kTlPartial = 1u << 27;
+constexpr int kMaxParts = 8;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;
@@ -91,6 +96,11 @@ struct Cfg {
 
 struct Params {
   int B, H, N, nQb, nKb, nQt, nPairs, nWork;
+  // Work units: items [0, split_first) whole, items [split_first, nWork) in split_parts parts of
+  // their key-block lists each (the last, partly filled wave of the persistent grid is cut finer).
+  int nUnits, split_first, split_parts;
+  float* part_o;    // [slot][2][128][D] unnormalised O of a partial unit, slot = (item - split_first) * parts + part
+  float2* part_ml;  // [slot][2][128] (reference max, row sum) of a partial unit
   const int32_t* offsets;
   const int32_t* kv_idx;
   void* o;
@@ -131,7 +141,7 @@ template <int NB>
 struct TileIter {
   const int32_t* idx;
   int pos[NB], end[NB], cur[NB], base[NB], win[NB];
-  int nKb, dense_j, lane;
+  int nKb, dense_j, lane, jhi;
   uint32_t dense_mask;
   bool dense;
   int* status;
@@ -156,13 +166,17 @@ struct TileIter {
     }
   }
 
+  // Part `part` of `parts` of the item's tiles: every index list (or the dense range) is cut by
+  // position into `parts` nearly equal pieces, so each (query block, key block) pair belongs to
+  // exactly one part.
   __device__ __forceinline__ void init(const Params& p, bool is_dense, int bh, int first_block,
-                                       int lane_id) {
+                                       int lane_id, int part, int parts) {
     idx = p.kv_idx;
     nKb = p.nKb;
     status = p.status;
     dense = is_dense;
-    dense_j = 0;
+    dense_j = (int)(((int64_t)p.nKb * part) / parts);
+    jhi = (int)(((int64_t)p.nKb * (part + 1)) / parts);
     dense_mask = 0;
     lane = lane_id;
     const int32_t nnz = is_dense ? 0 : __ldg(p.offsets + (int64_t)p.B * p.H * p.nQb);
@@ -179,8 +193,8 @@ struct TileIter {
           if (b < 0 || e < b || e > nnz || e - b > p.nKb) {
             report_error(status, LOSA_ERR_BAD_INDEX);
           } else {
-            pos[n] = b;
-            end[n] = e;
+            pos[n] = b + (int)(((int64_t)(e - b) * part) / parts);
+            end[n] = b + (int)(((int64_t)(e - b) * (part + 1)) / parts);
             refill(n);
             fetch(n);
           }
@@ -191,7 +205,7 @@ struct TileIter {
 
   __device__ __forceinline__ bool next(int& j, uint32_t& memb) {
     if (dense) {
-      if (dense_j >= nKb || dense_mask == 0) return false;
+      if (dense_j >= jhi || dense_mask == 0) return false;
       j = dense_j++;
       memb = dense_mask;
       return true;
@@ -350,7 +364,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       uint32_t nq[2] = {0, 0}, nk = 0, nv = 0, te = 0, ent;
       LOSA_TL_NEXT(ent);
       while ((ent >> 28) == 1) {
-        const int w = (int)(ent & 0x0fffffffu);
+        const int w = (int)(ent & kTlItemMask);
         const int bh = w / p.nPairs, pr = w % p.nPairs;
         const int b = bh / p.H, h = bh % p.H;
 #pragma unroll
@@ -431,6 +445,8 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       while ((ent >> 28) == 1) {
         bool q_ready = false, pend = false;
         uint32_t pend_vs = 0, pend_vph = 0, pv_item = 0;
+        // the producer loads this query tile for every item in which the tile exists
+        const bool q_loaded = 2 * ((int)(ent & kTlItemMask) % p.nPairs) + qt < p.nQt;
         for (;;) {
           LOSA_TL_NEXT(ent);
           const bool more = (ent >> 28) == 0;
@@ -526,7 +542,15 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if (leader) ptx::mma_commit(&ctl->o_done[qt]);  // every product of the item is done
           ++nof;
         }
-        if (q_ready && leader) ptx::mma_commit(&ctl->q_empty[qt]);
+        if (q_ready) {
+          if (leader) ptx::mma_commit(&ctl->q_empty[qt]);
+        } else if (q_loaded) {
+          // no key tile of this unit was listed by the query tile (a part of a short list can be
+          // empty): the query tile was loaded all the same and its buffer has to be handed back
+          LOSA_WAIT(&ctl->q_full[qt], nq & 1);
+          ++nq;
+          if (leader) ptx::mbar_arrive(&ctl->q_empty[qt]);
+        }
       }
     }
   } else if (warp == kSchedulerWarp) {
@@ -540,11 +564,21 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       int w = 0;
       if (lane == 0) w = atomicAdd(p.work_counter, 1);
       w = __shfl_sync(0xffffffffu, w, 0);
-      if (w >= p.nWork) break;
+      if (w >= p.nUnits) break;
+      // units past split_first are parts of the key range of the last items
+      int part = 0, parts = 1;
+      uint32_t flags = 0;
+      if (w >= p.split_first) {
+        const int r = w - p.split_first;
+        parts = p.split_parts;
+        part = r % parts;
+        w = p.split_first + r / parts;
+        flags = kTlPartial | ((uint32_t)part << 24);
+      }
       const int bh = w / p.nPairs, pr = w % p.nPairs;
-      LOSA_TL_PUT(kTlItem | (uint32_t)w);
+      LOSA_TL_PUT(kTlItem | flags | (uint32_t)w);
       TileIter<kNB> it;
-      it.init(p, MODE != kSparse, bh, 2 * pr * kQBT, lane);
+      it.init(p, MODE != kSparse, bh, 2 * pr * kQBT, lane, part, parts);
       int j;
       uint32_t memb;
       while (it.next(j, memb)) LOSA_TL_PUT((uint32_t)j | (memb << 16));
@@ -572,7 +606,9 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
     LOSA_TL_NEXT(ent);
     while ((ent >> 28) == 1) {
-      const int w = (int)(ent & 0x0fffffffu);
+      const int w = (int)(ent & kTlItemMask);
+      const bool partial = (ent & kTlPartial) != 0;
+      const int part = (int)((ent >> 24) & 7u);
       const int bh = w / p.nPairs, pr = w % p.nPairs;
       const int b = bh / p.H, h = bh % p.H;
       const int T = 2 * pr + qt;
@@ -703,6 +739,9 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const bool valid = grow < p.N;
           const float inv = (l > 0.f) ? 1.f / l : 0.f;
           const int64_t off = (int64_t)b * p.sb + (int64_t)h * p.sh + (int64_t)grow * p.sn;
+          const int64_t pslot =
+              ((((int64_t)(w - p.split_first) * p.split_parts + part) * 2 + qt) * 128 + row);
+          if (partial) p.part_ml[pslot] = make_float2(m_ref, l);
           if (pv_item > 0) {
             // o_done advances once per item, so its parity is unambiguous here (a product's own barrier may be
             // one, two or three phases from this warp's last look at it)
@@ -720,7 +759,14 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
               for (int c = 0; c < 32; ++c) r[c] = 0u;
             }
-            if (valid) {
+            if (partial) {
+              // a part of the key range: unnormalised O, merged with the other parts afterwards
+              float4* dst = reinterpret_cast<float4*>(p.part_o + pslot * D + c0);
+#pragma unroll
+              for (int c = 0; c < 32; c += 4)
+                dst[c >> 2] = make_float4(__uint_as_float(r[c]), __uint_as_float(r[c + 1]),
+                                          __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
+            } else if (valid) {
               if (p.o_f32) {
                 float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + off + c0);
 #pragma unroll
@@ -827,6 +873,73 @@ teardown:
 #undef LOSA_WAIT_RELAXED
 #undef LOSA_WAIT
 
+// Merge of the partial units: for every row of the split items, combine the parts' unnormalised
+// O, reference maximum and row sum (the usual log-sum-exp merge) and write the attention output.
+// grid = (split items, 2 query tiles), 4 warps; a warp takes 32 rows, its lanes the columns.
+template <int D>
+__global__ void __launch_bounds__(128) merge_parts_kernel(const Params p) {
+  const int r = blockIdx.x, qt = blockIdx.y;
+  const int w = p.split_first + r;
+  const int bh = w / p.nPairs, pr = w % p.nPairs;
+  const int T = 2 * pr + qt;
+  if (T >= p.nQt) return;
+  const int b = bh / p.H, h = bh % p.H;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int parts = p.split_parts;
+  for (int rr = 0; rr < 32; ++rr) {
+    const int row = warp * 32 + rr;
+    const int grow = T * 128 + row;
+    if (grow >= p.N) break;
+    float sc[kMaxParts];
+    float m = -INFINITY;
+#pragma unroll
+    for (int s = 0; s < kMaxParts; ++s) {
+      sc[s] = 0.f;
+      if (s < parts) {
+        const float2 ml = p.part_ml[(((int64_t)r * parts + s) * 2 + qt) * 128 + row];
+        if (ml.y > 0.f) m = fmaxf(m, ml.x);
+      }
+    }
+    float L = 0.f;
+#pragma unroll
+    for (int s = 0; s < kMaxParts; ++s) {
+      if (s < parts) {
+        const float2 ml = p.part_ml[(((int64_t)r * parts + s) * 2 + qt) * 128 + row];
+        if (ml.y > 0.f) {
+          sc[s] = ptx::ex2_approx(ml.x - m);
+          L += ml.y * sc[s];
+        }
+      }
+    }
+    const float inv = (L > 0.f) ? 1.f / L : 0.f;
+    const int d = lane * 4;
+    if (d < D) {
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int s = 0; s < kMaxParts; ++s) {
+        if (s < parts && sc[s] != 0.f) {
+          const float4 v = *reinterpret_cast<const float4*>(
+              p.part_o + ((((int64_t)r * parts + s) * 2 + qt) * 128 + row) * D + d);
+          acc.x += v.x * sc[s];
+          acc.y += v.y * sc[s];
+          acc.z += v.z * sc[s];
+          acc.w += v.w * sc[s];
+        }
+      }
+      const int64_t off = (int64_t)b * p.sb + (int64_t)h * p.sh + (int64_t)grow * p.sn + d;
+      if (p.o_f32) {
+        *reinterpret_cast<float4*>(static_cast<float*>(p.o) + off) =
+            make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+      } else {
+        uint2 v;
+        v.x = ptx::pack_bf16x2(acc.x * inv, acc.y * inv);
+        v.y = ptx::pack_bf16x2(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.o) + off) = v;
+      }
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------- host side
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
@@ -906,9 +1019,31 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
   }
   int sms = sm_count();
   if (sms <= 0) return LOSA_ERR_CUDA;
-  const int grid = min(min(sms, kMaxPersistentCtas), prm.nWork);
+  const int ctas = min(sms, kMaxPersistentCtas);
+  // The items of the last, partly filled wave of the persistent grid (all items, if there are
+  // fewer than CTAs) are cut into parts of the key range, so that the wave ends after 1/parts of
+  // an item; their partial results are merged by a second, small kernel.  Attention output
+  // only: the mass epilogue needs a row's final statistics inside the kernel.
+  prm.nUnits = prm.nWork;
+  prm.split_first = prm.nWork;
+  prm.split_parts = 1;
+  if ((MODE == kDense || MODE == kSparse) && prm.nWork <= (int)kTlItemMask) {
+    const int rest = (prm.nWork < ctas) ? prm.nWork : prm.nWork % ctas;
+    int parts = rest > 0 ? ctas / rest : 1;
+    parts = min(min(parts, kMaxParts), prm.nKb);
+    if (parts >= 2) {
+      prm.split_first = prm.nWork - rest;
+      prm.split_parts = parts;
+      prm.nUnits = prm.split_first + rest * parts;
+    }
+  }
+  const int grid = min(ctas, prm.nUnits);
   kern<<<grid, kThreads, smem, st>>>(mq, mk, mv, prm);
   LOSA_CUDA_TRY(cudaGetLastError());
+  if (prm.split_parts > 1) {
+    merge_parts_kernel<D><<<dim3(prm.nWork - prm.split_first, 2), 128, 0, st>>>(prm);
+    LOSA_CUDA_TRY(cudaGetLastError());
+  }
   return LOSA_OK;
 }
 
@@ -931,7 +1066,10 @@ extern "C" int losa_debug_trace(void* host, size_t bytes) {
 #endif
 
 size_t attn_workspace_bytes(AttnMode mode, const Geometry& g) {
-  if (mode == kDense || mode == kSparse) return kCounterBytes;
+  // attention output: counter, then one slot per partial unit (at most one per CTA) holding the
+  // rows' (max, sum) and unnormalised O of both query tiles
+  if (mode == kDense || mode == kSparse)
+    return kCounterBytes + kPartMlBytes + (size_t)kMaxPersistentCtas * 2 * 128 * (size_t)g.D * sizeof(float);
   // counter, per-CTA row statistics, per-CTA table of one entry per row and key tile
   return kCounterBytes + kRowstatBytes +
          (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2);
@@ -963,6 +1101,8 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
   prm.rowstat = reinterpret_cast<float2*>(static_cast<char*>(ws) + kCounterBytes);
   prm.table = reinterpret_cast<float2*>(static_cast<char*>(ws) + kCounterBytes +
                                         ((mode == kMass || mode == kFused) ? kRowstatBytes : 0));
+  prm.part_ml = reinterpret_cast<float2*>(static_cast<char*>(ws) + kCounterBytes);
+  prm.part_o = reinterpret_cast<float*>(static_cast<char*>(ws) + kCounterBytes + kPartMlBytes);
   prm.scale_log2 = g.scale * kLog2e;
   prm.status = status_word_device();
   if (!prm.status) return LOSA_ERR_CUDA;

@@ -22,6 +22,8 @@ def sample_rows(wl, n, seed):
     ids = set(rng.choice(wl.rows, size=n, replace=False).tolist())
     ids.add(wl.nQb - 1)             # ragged last query block of the first head
     ids.add(wl.rows - wl.nQb)       # first query block of the last head
+    ids.add(wl.rows - 1)            # ragged last query block of the last head: its work item is one of
+    ids.add(wl.rows - 3)            # those the attention kernel cuts into parts and merges afterwards
     return np.array(sorted(ids), dtype=np.int32)
 
 
@@ -119,7 +121,9 @@ def test_full_size_parity_on_sampled_query_blocks(name, n_sample):
         o_f, mass_f = losa.losa_attn_mass(qd, kd, vd, wl.R, wl.C, out_dtype=torch.float32)
         o_d = losa.losa_attn(qd, kd, vd, wl.R, wl.C, out_dtype=torch.float32)
         losa.check_async("fused construction")
-        assert torch.equal(o_f, o_d)
+        # the attention-only call cuts its last work items into parts and merges them: same result up
+        # to the summation order
+        assert (o_f - o_d).abs().max().item() <= util.MAX_ABS_TOL
         gmf = mass_f.cpu().numpy().reshape(wl.rows, wl.nKb)
         assert float(np.abs(gmf[ids] - ref_mass).max()) <= util.MASS_TOL
         assert np.abs(gmf.astype(np.float64).sum(1) - 1.0).max() <= util.MASS_TOL
