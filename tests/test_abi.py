@@ -33,7 +33,8 @@ def test_workspace_sizing_and_status_strings_need_no_gpu():
     p = binding.Problem(1, 12, 32760, 128, 128, 128, 12 * 32760 * 128, 32760 * 128, 128, 0.0)
     assert binding.losa_workspace_bytes(binding.LOSA_OP_BLOCK_MASS, p) > 0
     assert binding.losa_workspace_bytes(binding.LOSA_OP_SELECT, p) > 0
-    assert 0 < binding.losa_workspace_bytes(binding.LOSA_OP_ATTN, p) <= 4096
+    # counter + one partial-result slot per persistent CTA: independent of N
+    assert 0 < binding.losa_workspace_bytes(binding.LOSA_OP_ATTN, p) <= 32 << 20
     bad = binding.Problem(1, 1, 128, 96, 128, 128, 128 * 96, 128 * 96, 96, 0.0)
     assert binding.losa_workspace_bytes(binding.LOSA_OP_BLOCK_MASS, bad) == 0
     assert binding.losa_status_string(0) == "LOSA_OK"
