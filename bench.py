@@ -41,8 +41,18 @@ UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one sparse-forward launch, from the ncu capture
 # summarised in profiles/losa_attn_kernel_wan_ncu.md (not re-measured by this script)
-NCU_DRAM_BYTES_PER_LAUNCH = {"wan": 0.304484e9 + 0.083875e9}
+NCU_DRAM_BYTES_PER_LAUNCH = {"wan": 0.304626e9 + 0.085013e9}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def merge_kernel_runs(wl) -> bool:
+    """Whether the attention-only calls launch their second (merge) kernel for this shape: the host
+    rule of the library, restated (work items = pairs of 128-row query tiles per head)."""
+    ctas = min(torch.cuda.get_device_properties(0).multi_processor_count, 160)
+    n_work = wl.B * wl.H * ((-(-wl.N // 128) + 1) // 2)
+    rest = n_work if n_work < ctas else n_work % ctas
+    parts = min(ctas // rest, 8, -(-wl.N // wl.C)) if rest else 1
+    return parts >= 2
 
 
 def parse_args():
@@ -474,7 +484,9 @@ def main():
             "algorithmic_bytes_per_launch": 4 * q0.numel() * 2,
         },
         "clocks": clocks.summary(),
-        "gpu_launches": args.steps * (1 + 3 + args.draws + 1 + 1),
+        # per step: mass 1, select 3, sparse `draws`, dense 1, fused 1; each attention-only call adds
+        # its merge kernel when the last wave of work items is cut into parts
+        "gpu_launches": args.steps * (1 + 3 + (args.draws + 1) * (2 if merge_kernel_runs(wl) else 1) + 1),
     }
     if e2e is not None:
         line["e2e"] = e2e

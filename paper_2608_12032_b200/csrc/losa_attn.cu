@@ -875,10 +875,11 @@ teardown:
 
 // Merge of the partial units: for every row of the split items, combine the parts' unnormalised
 // O, reference maximum and row sum (the usual log-sum-exp merge) and write the attention output.
-// grid = (split items, 2 query tiles), 4 warps; a warp takes 32 rows, its lanes the columns.
+// grid = (split items, 2 query tiles x 8 row chunks), 4 warps; a warp takes 4 rows, its lanes the
+// columns.
 template <int D>
 __global__ void __launch_bounds__(128) merge_parts_kernel(const Params p) {
-  const int r = blockIdx.x, qt = blockIdx.y;
+  const int r = blockIdx.x, qt = blockIdx.y >> 3, chunk = blockIdx.y & 7;
   const int w = p.split_first + r;
   const int bh = w / p.nPairs, pr = w % p.nPairs;
   const int T = 2 * pr + qt;
@@ -886,8 +887,9 @@ __global__ void __launch_bounds__(128) merge_parts_kernel(const Params p) {
   const int b = bh / p.H, h = bh % p.H;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int parts = p.split_parts;
-  for (int rr = 0; rr < 32; ++rr) {
-    const int row = warp * 32 + rr;
+#pragma unroll
+  for (int rr = 0; rr < 4; ++rr) {
+    const int row = chunk * 16 + warp * 4 + rr;
     const int grow = T * 128 + row;
     if (grow >= p.N) break;
     float sc[kMaxParts];
@@ -1041,7 +1043,7 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
   kern<<<grid, kThreads, smem, st>>>(mq, mk, mv, prm);
   LOSA_CUDA_TRY(cudaGetLastError());
   if (prm.split_parts > 1) {
-    merge_parts_kernel<D><<<dim3(prm.nWork - prm.split_first, 2), 128, 0, st>>>(prm);
+    merge_parts_kernel<D><<<dim3(prm.nWork - prm.split_first, 16), 128, 0, st>>>(prm);
     LOSA_CUDA_TRY(cudaGetLastError());
   }
   return LOSA_OK;
