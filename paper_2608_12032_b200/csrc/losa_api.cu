@@ -49,7 +49,10 @@ int make_geometry(const losa_problem_t* p, Geometry* g) {
   if (!p) return LOSA_ERR_INVALID_ARG;
   if (p->B <= 0 || p->H <= 0 || p->N <= 0) return LOSA_ERR_INVALID_ARG;
   if (!(p->D == 64 || p->D == 128)) return LOSA_ERR_UNSUPPORTED;
-  if (!((p->R == 64 && p->C == 64) || (p->R == 128 && p->C == 128))) return LOSA_ERR_UNSUPPORTED;
+  // query blocks of 64 or 128 rows; key blocks of 32, 64 or 128 rows, gathered into 128-key tiles
+  if (!((p->R == 64 && p->C == 64) || (p->R == 128 && (p->C == 128 || p->C == 64 || p->C == 32))))
+    return LOSA_ERR_UNSUPPORTED;
+  if ((int64_t)(p->N + p->C - 1) / p->C >= 0xffff) return LOSA_ERR_UNSUPPORTED;  // 16-bit block index in the tile list
   if (p->sn < p->D || p->sh <= 0 || p->sb <= 0) return LOSA_ERR_INVALID_ARG;
   if ((p->sn % 8) || (p->sh % 8) || (p->sb % 8)) return LOSA_ERR_INVALID_ARG;
   if (!(p->scale >= 0.0f) || isinf(p->scale)) return LOSA_ERR_INVALID_ARG;

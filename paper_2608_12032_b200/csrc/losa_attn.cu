@@ -62,35 +62,42 @@ constexpr uint32_t kTlItem = 1u << 28, kTlEnd = 2u << 28;  // entry type in bits
 // An item header carries the work item in bits 23:0 and, for a unit that covers only part of the
 // item's key range, the part index in bits 26:24 and a flag in bit 27.
 constexpr uint32_t kTlItemMask = 0x00ffffffu, kTlPartial = 1u << 27;
+// A K/V tile is a group of 128 / C consecutive tile entries (key block index in bits 15:0,
+// membership bits from bit 16); the last group of an item is padded with this entry: no member,
+// and a block index whose rows lie past the end of the tensor (the copy engine fills zeros).
+constexpr uint32_t kTlPad = 0xffffu;
 constexpr int kMaxParts = 8;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;
 
-template <int D, int BLK, int MODE>
+template <int D, int R, int C_, int MODE, int KT>
 struct Cfg {
-  static constexpr int kC = BLK;                      // keys per K/V tile
-  static constexpr int kQBT = 128 / BLK;              // query blocks per 128-row tile
+  static constexpr int kC = C_;                       // keys per key block
+  static constexpr int kT = KT;                       // keys per K/V tile: one S = Q K^T per tile
+  static constexpr int kG = kT / kC;                  // key blocks gathered into one K/V tile
+  static constexpr int kQBT = 128 / R;                // query blocks per 128-row tile
   static constexpr int kNB = 2 * kQBT;                // query blocks per work item
   static constexpr int kDH = D / 64;                  // 64-element slabs along D
   static constexpr int kQSlab = 128 * 128;            // bytes of a [128][64] bf16 slab
   static constexpr int kQBytes = kDH * kQSlab;        // one query tile
-  static constexpr int kKVSlab = kC * 128;            // bytes of a [C][64] bf16 slab
+  static constexpr int kKVSlab = kT * 128;            // bytes of a [128][64] bf16 slab
   static constexpr int kKVBytes = kDH * kKVSlab;      // one K (or V) tile
+  static constexpr int kBoxBytes = kC * 128;          // one key block of a slab (a TMA box)
   static constexpr bool kHasV = (MODE != kMass);
   static constexpr bool kWantMass = (MODE == kMass || MODE == kFused);
-  static constexpr int kW = kC;                       // columns of S: one K/V tile per S = Q K^T
-  // TMEM (512 columns): with an O accumulator, per query tile one S of up to 128 columns (P in
-  // place) and O; the mass pass has no O and double-buffers S instead.
+  static constexpr int kW = kT;                       // columns of S
+  // TMEM (512 columns): with an O accumulator, per query tile one S of 128 columns (P in place)
+  // and O; the mass pass has no O and double-buffers S instead.
   static constexpr int kNS = kHasV ? 1 : 2;           // S buffers per query tile
   static constexpr int kSStride = kHasV ? 128 : 256;  // TMEM columns between the tiles' S areas
   static constexpr int kRingBudget = (kHasV ? 160 : 128) * 1024;  // K + V rings
-  // a V tile stays in use about one tile longer than a K tile (its products are issued one
-  // sub-tile behind), so V gets the deeper ring
+  // a V tile stays in use about one tile longer than a K tile (its product is issued after the
+  // tile's softmax), so V gets the deeper ring
   static constexpr int kNV = kHasV ? ((kKVBytes >= 32768) ? 3 : 4) : 0;
   static constexpr int kNK0 = (kRingBudget - kNV * kKVBytes) / kKVBytes;
   static constexpr int kNK = kNK0 > 6 ? 6 : kNK0;
-  static constexpr uint32_t kIdescQK = ptx::idesc_bf16_f32(128, kW, false, false);  // one sub-tile
+  static constexpr uint32_t kIdescQK = ptx::idesc_bf16_f32(128, kW, false, false);
   static constexpr uint32_t kIdescPV = ptx::idesc_bf16_f32(128, D, false, true);
 };
 
@@ -274,6 +281,17 @@ __device__ unsigned long long g_trace[8][4096];
     ++te;                                                                            \
   } while (0)
 
+// Next K/V tile of the tile list: its kG entries into grp[]; `more` is false (and grp[0] holds the
+// entry) when the item ends instead.
+#define LOSA_TL_NEXT_TILE(grp, more)                            \
+  do {                                                          \
+    LOSA_TL_NEXT((grp)[0]);                                     \
+    (more) = ((grp)[0] >> 28) == 0;                             \
+    if (more) {                                                 \
+      _Pragma("unroll") for (int g_ = 1; g_ < kG; ++g_) LOSA_TL_NEXT((grp)[g_]); \
+    }                                                           \
+  } while (0)
+
 // Scheduler side: append one entry (whole warp; lane 0 writes).
 #define LOSA_TL_PUT(ent)                                                             \
   do {                                                                               \
@@ -288,13 +306,13 @@ __device__ unsigned long long g_trace[8][4096];
     ++te;                                                                            \
   } while (0)
 
-template <int D, int BLK, int MODE>
+template <int D, int R, int C_, int MODE, int KT>
 __global__ void __launch_bounds__(kThreads, 1)
 losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, const Params p) {
-  using C = Cfg<D, BLK, MODE>;
+  using C = Cfg<D, R, C_, MODE, KT>;
   using Ctl = Control<C::kNK, C::kNV>;
-  constexpr int kC = C::kC, kQBT = C::kQBT, kNB = C::kNB, kW = C::kW, kNS = C::kNS;
+  constexpr int kC = C::kC, kG = C::kG, kQBT = C::kQBT, kNB = C::kNB, kW = C::kW, kNS = C::kNS;
   constexpr uint32_t kSStride = C::kSStride, kNVs = C::kNV > 0 ? C::kNV : 1;
   constexpr uint32_t kQMask = (1u << kQBT) - 1u;
 
@@ -383,28 +401,48 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
         }
         for (;;) {
-          LOSA_TL_NEXT(ent);
-          if ((ent >> 28) != 0) break;
-          const int j = (int)(ent & 0xffffu);
+          uint32_t grp[kG];
+          bool more;
+          LOSA_TL_NEXT_TILE(grp, more);
+          if (!more) {
+            ent = grp[0];
+            break;
+          }
+          // a tile gathers kG key blocks: block g of the group goes to rows g * C ... of the stage
+          // (a padding entry names rows past the end of the tensor, which are filled with zeros)
           const uint32_t ks = nk % C::kNK;
           LOSA_WAIT_RELAXED(&ctl->k_empty[ks], ((nk / C::kNK) & 1) ^ 1);
-          if (lane == 0) {
-            ptx::mbar_arrive_expect_tx(&ctl->k_full[ks], C::kKVBytes);
+          // one copy per (key block, slab), issued by as many lanes at once: a single thread
+          // issuing 8 or 16 small copies per tile cannot keep up with the tile rate
+          if (lane == 0) ptx::mbar_arrive_expect_tx(&ctl->k_full[ks], C::kKVBytes);
+          __syncwarp();
+          if (lane < kG * C::kDH) {
+            const int g = lane / C::kDH, s = lane % C::kDH;
+            uint32_t eg = grp[0];
 #pragma unroll
-            for (int s = 0; s < C::kDH; ++s)
-              ptx::tma_load_4d(sK + ks * C::kKVBytes + s * C::kKVSlab, &map_k, &ctl->k_full[ks],
-                               s * 64, j * kC, h, b);
+            for (int gg = 1; gg < kG; ++gg)
+              if (g == gg) eg = grp[gg];
+            const int jg = (int)(eg & 0xffffu);
+            const int r0 = (jg == (int)kTlPad) ? p.nKb * kC : jg * kC;
+            ptx::tma_load_4d(sK + ks * C::kKVBytes + s * C::kKVSlab + g * C::kBoxBytes, &map_k,
+                             &ctl->k_full[ks], s * 64, r0, h, b);
           }
           ++nk;
           if (C::kHasV) {
             const uint32_t vs = nv % kNVs;
             LOSA_WAIT_RELAXED(&ctl->v_empty[vs], ((nv / kNVs) & 1) ^ 1);
-            if (lane == 0) {
-              ptx::mbar_arrive_expect_tx(&ctl->v_full[vs], C::kKVBytes);
+            if (lane == 0) ptx::mbar_arrive_expect_tx(&ctl->v_full[vs], C::kKVBytes);
+            __syncwarp();
+            if (lane < kG * C::kDH) {
+              const int g = lane / C::kDH, s = lane % C::kDH;
+              uint32_t eg = grp[0];
 #pragma unroll
-              for (int s = 0; s < C::kDH; ++s)
-                ptx::tma_load_4d(sV + vs * C::kKVBytes + s * C::kKVSlab, &map_v, &ctl->v_full[vs],
-                                 s * 64, j * kC, h, b);
+              for (int gg = 1; gg < kG; ++gg)
+                if (g == gg) eg = grp[gg];
+              const int jg = (int)(eg & 0xffffu);
+              const int r0 = (jg == (int)kTlPad) ? p.nKb * kC : jg * kC;
+              ptx::tma_load_4d(sV + vs * C::kKVBytes + s * C::kKVSlab + g * C::kBoxBytes, &map_v,
+                               &ctl->v_full[vs], s * 64, r0, h, b);
             }
             ++nv;
           }
@@ -448,9 +486,17 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // the producer loads this query tile for every item in which the tile exists
         const bool q_loaded = 2 * ((int)(ent & kTlItemMask) % p.nPairs) + qt < p.nQt;
         for (;;) {
-          LOSA_TL_NEXT(ent);
-          const bool more = (ent >> 28) == 0;
-          const uint32_t memb = (ent >> 16) & 0xfu;
+          uint32_t grp[kG];
+          bool more;
+          LOSA_TL_NEXT_TILE(grp, more);
+          if (!more) ent = grp[0];
+          // the query tile takes part in a K/V tile if any of its query blocks lists any of the
+          // tile's key blocks
+          uint32_t memb = 0;
+          if (more) {
+#pragma unroll
+            for (int g = 0; g < kG; ++g) memb |= (grp[g] >> 16) & 0xfu;
+          }
           const uint32_t ks = nt % C::kNK, kph = (nt / C::kNK) & 1;
           const uint32_t vs = nt % kNVs, vph = (nt / kNVs) & 1;
           const bool member = more && ((memb >> (qt * kQBT)) & kQMask) != 0;
@@ -579,9 +625,17 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       LOSA_TL_PUT(kTlItem | flags | (uint32_t)w);
       TileIter<kNB> it;
       it.init(p, MODE != kSparse, bh, 2 * pr * kQBT, lane, part, parts);
-      int j;
+      int j, emitted = 0;
       uint32_t memb;
-      while (it.next(j, memb)) LOSA_TL_PUT((uint32_t)j | (memb << 16));
+      while (it.next(j, memb)) {
+        LOSA_TL_PUT((uint32_t)j | (memb << 16));
+        ++emitted;
+      }
+      // K/V tiles are groups of kG entries: pad the item's last group
+      while (emitted % kG != 0) {
+        LOSA_TL_PUT(kTlPad);
+        ++emitted;
+      }
     }
     LOSA_TL_PUT(kTlEnd);
     if ((te & 31) != 0) {  // publish the last, partly filled chunk
@@ -597,9 +651,8 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t lane_base = (uint32_t)(wl * 32) << 16;
     const uint32_t tS = tmem_base + lane_base + qt * kSStride;  // P overwrites its first kW/2 columns
     const uint32_t tO = tmem_base + lane_base + 256 + qt * 128;
-    const int sub = (BLK == 64) ? (wl >> 1) : 0;
+    const int sub = (R == 64) ? (wl >> 1) : 0;
     const int my_bit = qt * kQBT + sub;
-    const int tail = p.N - (p.nKb - 1) * kC;  // valid keys of the last K/V tile
     uint32_t nsub = 0, nwg = 0, nod = 0;      // nsub: key tiles of this query tile so far
     uint32_t te = 0, ent;
     TR_DECL((wl == 0) ? qt : 7);
@@ -619,12 +672,27 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (C::kWantMass)
         tab = p.table + ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * 128 + row;
       for (;;) {
-        LOSA_TL_NEXT(ent);
-        if ((ent >> 28) != 0) break;
-        const int j = (int)(ent & 0xffffu);
-        const uint32_t memb = (ent >> 16) & 0xfu;
+        uint32_t grp[kG];
+        bool more;
+        LOSA_TL_NEXT_TILE(grp, more);
+        if (!more) {
+          ent = grp[0];
+          break;
+        }
+        // vc[g]: how many keys of key block g of the tile this row attends to: all that exist, if
+        // the row's query block lists the block, none otherwise (nor for a padding entry)
+        uint32_t memb = 0;
+        int vc[kG];
+        bool mine = false, full = true;
+#pragma unroll
+        for (int g = 0; g < kG; ++g) {
+          memb |= (grp[g] >> 16) & 0xfu;
+          const int jg = (int)(grp[g] & 0xffffu);
+          vc[g] = ((grp[g] >> (16 + my_bit)) & 1u) ? min(kC, p.N - jg * kC) : 0;
+          mine = mine || vc[g] > 0;
+          full = full && vc[g] == kC;
+        }
         if (((memb >> (qt * kQBT)) & kQMask) == 0) continue;
-        const bool mine = (memb >> my_bit) & 1u;
         const uint32_t buf = nsub % kNS;
         const uint32_t tSb = tS + buf * 128;
         // S of this key tile is complete, and so is every earlier product into O
@@ -646,10 +714,14 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if (lane == 0) ptx::mbar_arrive(&ctl->s_free[qt][buf]);
         }
         if (mine) {
-          if (j == p.nKb - 1 && tail < kW) {  // keys >= N do not exist
+          // Keys that do not exist (>= N) and key blocks the row's query block does not list get
+          // a score of -inf: they drop out of the maximum and their p is exactly 0.  Straight-line
+          // code over all 128 columns is faster than skipping blocks (measured: branches between
+          // the blocks cost the softmax 0.9 k cycles per tile at C = 32).
+          if (!full) {
 #pragma unroll
             for (int c = 0; c < kW; ++c)
-              if (c >= tail) sr[c] = 0xff800000u;
+              if ((c % kC) >= vc[c / kC]) sr[c] = 0xff800000u;
           }
           float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
           float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
@@ -693,7 +765,10 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           TR(5, nsub);
           const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
           const float2 nm2 = make_float2(-m_ref, -m_ref);
-          float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+          // (row sums per key block: the mass pass needs them apart; two chains per block)
+          float2 acc[kG][2];
+#pragma unroll
+          for (int g = 0; g < kG; ++g) acc[g][0] = acc[g][1] = make_float2(0.f, 0.f);
 #pragma unroll
           for (int c = 0; c < kW; c += 4) {
             float2 x0 = ptx::fma2(
@@ -704,18 +779,34 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             x0.y = ptx::ex2_approx(x0.y);
             x1.x = ptx::ex2_approx(x1.x);
             x1.y = ptx::ex2_approx(x1.y);
-            acc0 = ptx::add2(acc0, x0);
-            acc1 = ptx::add2(acc1, x1);
-            sr[c >> 1] = ptx::pack_bf16x2(x0.x, x0.y);
-            sr[(c >> 1) + 1] = ptx::pack_bf16x2(x1.x, x1.y);
-            if (C::kHasV && (c & 63) == 60) ptx::tmem_st32(tSb + (c >> 6) * 32, &sr[(c >> 6) * 32]);
+            acc[c / kC][0] = ptx::add2(acc[c / kC][0], x0);
+            acc[c / kC][1] = ptx::add2(acc[c / kC][1], x1);
+            if (C::kHasV) {
+              sr[c >> 1] = ptx::pack_bf16x2(x0.x, x0.y);
+              sr[(c >> 1) + 1] = ptx::pack_bf16x2(x1.x, x1.y);
+              // 64 keys of P are complete: store them while the rest is computed
+              if ((c & 63) == 60) ptx::tmem_st32(tSb + (c >> 6) * 32, &sr[(c >> 6) * 32]);
+            }
           }
           TR(6, nsub);
-          const float tsum = (acc0.x + acc0.y) + (acc1.x + acc1.y);
+          float gsum[kG], tsum = 0.f;
+#pragma unroll
+          for (int g = 0; g < kG; ++g) {
+            gsum[g] = (acc[g][0].x + acc[g][0].y) + (acc[g][1].x + acc[g][1].y);
+            tsum += gsum[g];
+          }
           l += tsum;
-          if (C::kWantMass) tab[(int64_t)j * 128] = make_float2(tsum, m_ref);
+          if (C::kWantMass) {
+            // one table entry per key block
+#pragma unroll
+            for (int g = 0; g < kG; ++g) {
+              if (vc[g] > 0) {
+                tab[(int64_t)(grp[g] & 0xffffu) * 128] = make_float2(gsum[g], m_ref);
+              }
+            }
+          }
         } else if (C::kHasV) {
-          // this half of the 128-row tile does not list the key block: P = 0
+          // this part of the 128-row tile lists none of the tile's key blocks: P = 0
           uint32_t z[32];
 #pragma unroll
           for (int c = 0; c < 32; ++c) z[c] = 0u;
@@ -823,7 +914,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               const float2 tv = tb[(int64_t)u * 128 + r];
               const float wgt =
                   (st[rr].y > 0.f) ? tv.x * ptx::ex2_approx(tv.y - st[rr].x) * st[rr].y : 0.f;
-              acc[(rr * 32) / BLK] += wgt;
+              acc[(rr * 32) / R] += wgt;
             }
 #pragma unroll
             for (int q = 0; q < kQBT; ++q) {
@@ -832,7 +923,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
               const int g = T * kQBT + q;
               if (lane == 0 && g < p.nQb) {
-                const int nvalid = min(BLK, p.N - g * BLK);
+                const int nvalid = min(R, p.N - g * R);
                 p.mass[((int64_t)bh * p.nQb + g) * p.nKb + u] = a / (float)nvalid;
               }
             }
@@ -868,6 +959,7 @@ teardown:
   }
 }
 
+#undef LOSA_TL_NEXT_TILE
 #undef LOSA_TL_NEXT
 #undef LOSA_TL_PUT
 #undef LOSA_WAIT_RELAXED
@@ -994,10 +1086,10 @@ int sm_count() {
   return n;
 }
 
-template <int D, int BLK, int MODE>
+template <int D, int R, int C_, int MODE, int KT>
 int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Params prm,
              cudaStream_t st) {
-  using C = Cfg<D, BLK, MODE>;
+  using C = Cfg<D, R, C_, MODE, KT>;
   using Ctl = Control<C::kNK, C::kNV>;
   CUtensorMap mq, mk, mv;
   int rc;
@@ -1006,7 +1098,7 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
   if ((rc = make_map(&mv, C::kHasV ? v : k, g, C::kC)) != LOSA_OK) return rc;
   const size_t smem =
       1024 + 2 * C::kQBytes + (size_t)(C::kNK + C::kNV) * C::kKVBytes + sizeof(Ctl);
-  auto kern = losa_attn_kernel<D, BLK, MODE>;
+  auto kern = losa_attn_kernel<D, R, C_, MODE, KT>;
   static bool configured = false;
   if (!configured) {
     // the in-kernel register reallocation must fit the registers the CTA is launched with
@@ -1052,10 +1144,23 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
 template <int MODE>
 int dispatch(const Geometry& g, const void* q, const void* k, const void* v, const Params& prm,
              cudaStream_t st) {
-  if (g.D == 128 && g.R == 128) return launch_t<128, 128, MODE>(g, q, k, v, prm, st);
-  if (g.D == 64 && g.R == 64) return launch_t<64, 64, MODE>(g, q, k, v, prm, st);
-  if (g.D == 128 && g.R == 64) return launch_t<128, 64, MODE>(g, q, k, v, prm, st);
-  if (g.D == 64 && g.R == 128) return launch_t<64, 128, MODE>(g, q, k, v, prm, st);
+  // K/V tiles of 128 keys (128 / C gathered key blocks, 128-wide MMAs) everywhere but in the
+  // sparse forward with 64 x 64 blocks: a 128-row query tile then spans two query blocks and a
+  // 128-key tile two key blocks, and with four index lists per work item nearly every tile is
+  // visited by somebody while half of its rows sit idle (measured at the CogVideoX shape:
+  // 7.34 ms with 128-key tiles, 6.86 ms with 64-key tiles).
+#define LOSA_CASE(d, r, c)                                                          \
+  if (g.D == d && g.R == r && g.C == c)                                             \
+  return launch_t<d, r, c, MODE, (r == 64 && c == 64 && MODE == kSparse) ? 64 : 128>(g, q, k, v, prm, st)
+  LOSA_CASE(128, 128, 128);
+  LOSA_CASE(64, 64, 64);
+  LOSA_CASE(128, 128, 32);  // the paper's own block geometry
+  LOSA_CASE(64, 128, 32);
+  LOSA_CASE(128, 64, 64);
+  LOSA_CASE(64, 128, 128);
+  LOSA_CASE(128, 128, 64);
+  LOSA_CASE(64, 128, 64);
+#undef LOSA_CASE
   return LOSA_ERR_UNSUPPORTED;
 }
 

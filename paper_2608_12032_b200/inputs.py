@@ -81,6 +81,8 @@ WORKLOADS: Dict[str, Workload] = {
     "cogvideox": Workload("cogvideox", 1, 48, 64, (13, 30, 45), 226, 64, 64),
     "wan": Workload("wan", 1, 12, 128, (21, 30, 52), 0, 128, 128),
     "hunyuan": Workload("hunyuan", 1, 24, 128, (33, 45, 80), 0, 128, 128),
+    # the Wan-shaped layer with the paper's own block geometry (query blocks of 128, key blocks of 32)
+    "wan_r128c32": Workload("wan_r128c32", 1, 12, 128, (21, 30, 52), 0, 128, 32),
 }
 
 
