@@ -34,7 +34,8 @@
  *    that overflowed its capacity) are recorded in a status word that
  *    losa_async_status() returns and clears.  No kernel ever traps, asserts
  *    or waits without a bound.
- *  - Supported shapes: D in {64, 128}; (R, C) in {(64, 64), (128, 128)}.
+ *  - Supported shapes: D in {64, 128}; (R, C) in {(64, 64), (128, 128), (128, 64), (128, 32)}
+ *    (the last is the block geometry the paper runs with); fewer than 65535 key blocks.
  */
 #ifndef LOSA_H_
 #define LOSA_H_
@@ -70,7 +71,7 @@ enum { LOSA_DTYPE_BF16 = 0, LOSA_DTYPE_F32 = 1 };
 
 typedef struct {
   int32_t B, H, N, D; /* batch, heads, VALID tokens, head dimension                     */
-  int32_t R, C;       /* query / key-value block size                                   */
+  int32_t R, C;       /* query / key-value block size: (64,64), (128,128), (128,64), (128,32) */
   int64_t sb, sh, sn; /* element strides of batch, head, token (D is contiguous)        */
   float scale;        /* softmax scale; 0 selects 1/sqrt(D) as in A = softmax(QK^T/sqrt d) */
 } losa_problem_t;
