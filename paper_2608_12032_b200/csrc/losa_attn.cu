@@ -106,6 +106,11 @@ struct Params {
   // Work units: items [0, split_first) whole, items [split_first, nWork) in split_parts parts of
   // their key-block lists each (the last, partly filled wave of the persistent grid is cut finer).
   int nUnits, split_first, split_parts;
+  // Sparse mode: the merged tile lists of all units, built by build_tile_lists_kernel before the
+  // attention kernel: unit u owns tl_entries[u * tl_cap ...], tl_count[u] of them (padded to whole tiles).
+  uint32_t* tl_entries;
+  int32_t* tl_count;
+  int tl_cap;
   float* part_o;    // [slot][2][128][D] unnormalised O of a partial unit, slot = (item - split_first) * parts + part
   float2* part_ml;  // [slot][2][128] (reference max, row sum) of a partial unit
   const int32_t* offsets;
@@ -137,102 +142,6 @@ struct Control {
   uint32_t tmem_base;
   uint32_t mma_lock;  // held while a burst of MMAs is issued
   int abort_flag;
-};
-
-// Ascending merge of the block-index lists of the (up to NB) query blocks of a work item.
-// Every role walks its own copy; the sequence is a pure function of the CSR, so they agree.
-// The whole warp walks it together: each lane keeps one entry of a 32-entry window per list
-// (one coalesced load per 32 tiles) and the current entry is broadcast with a shuffle, so no
-// role waits on a dependent global load per tile.  All 32 lanes must call every method.
-template <int NB>
-struct TileIter {
-  const int32_t* idx;
-  int pos[NB], end[NB], cur[NB], base[NB], win[NB];
-  int nKb, dense_j, lane, jhi;
-  uint32_t dense_mask;
-  bool dense;
-  int* status;
-
-  __device__ __forceinline__ void refill(int n) {
-    base[n] = pos[n];
-    const int at = pos[n] + lane;
-    win[n] = (at < end[n]) ? __ldg(idx + at) : INT_MAX;
-  }
-
-  __device__ __forceinline__ void fetch(int n) {
-    cur[n] = INT_MAX;
-    while (pos[n] < end[n]) {
-      if (pos[n] - base[n] >= 32) refill(n);
-      const int v = __shfl_sync(0xffffffffu, win[n], pos[n] - base[n]);
-      if ((unsigned)v < (unsigned)nKb) {
-        cur[n] = v;
-        return;
-      }
-      report_error(status, LOSA_ERR_BAD_INDEX);  // skipped, never used as an address
-      ++pos[n];
-    }
-  }
-
-  // Part `part` of `parts` of the item's tiles: every index list (or the dense range) is cut by
-  // position into `parts` nearly equal pieces, so each (query block, key block) pair belongs to
-  // exactly one part.
-  __device__ __forceinline__ void init(const Params& p, bool is_dense, int bh, int first_block,
-                                       int lane_id, int part, int parts) {
-    idx = p.kv_idx;
-    nKb = p.nKb;
-    status = p.status;
-    dense = is_dense;
-    dense_j = (int)(((int64_t)p.nKb * part) / parts);
-    jhi = (int)(((int64_t)p.nKb * (part + 1)) / parts);
-    dense_mask = 0;
-    lane = lane_id;
-    const int32_t nnz = is_dense ? 0 : __ldg(p.offsets + (int64_t)p.B * p.H * p.nQb);
-#pragma unroll
-    for (int n = 0; n < NB; ++n) {
-      const int g = first_block + n;
-      pos[n] = end[n] = base[n] = 0;
-      cur[n] = win[n] = INT_MAX;
-      if (g < p.nQb) {
-        dense_mask |= 1u << n;
-        if (!is_dense) {
-          const int64_t row = (int64_t)bh * p.nQb + g;
-          const int32_t b = __ldg(p.offsets + row), e = __ldg(p.offsets + row + 1);
-          if (b < 0 || e < b || e > nnz || e - b > p.nKb) {
-            report_error(status, LOSA_ERR_BAD_INDEX);
-          } else {
-            pos[n] = b + (int)(((int64_t)(e - b) * part) / parts);
-            end[n] = b + (int)(((int64_t)(e - b) * (part + 1)) / parts);
-            refill(n);
-            fetch(n);
-          }
-        }
-      }
-    }
-  }
-
-  __device__ __forceinline__ bool next(int& j, uint32_t& memb) {
-    if (dense) {
-      if (dense_j >= jhi || dense_mask == 0) return false;
-      j = dense_j++;
-      memb = dense_mask;
-      return true;
-    }
-    int m = INT_MAX;
-#pragma unroll
-    for (int n = 0; n < NB; ++n) m = min(m, cur[n]);
-    if (m == INT_MAX) return false;
-    memb = 0;
-#pragma unroll
-    for (int n = 0; n < NB; ++n) {
-      if (cur[n] == m) {
-        memb |= 1u << n;
-        ++pos[n];
-        fetch(n);
-      }
-    }
-    j = m;
-    return true;
-  }
 };
 
 // Event trace (diagnostic builds only, -DLOSA_TRACE): CTA 0 records (clock, event, counter) per role.
@@ -290,6 +199,26 @@ __device__ unsigned long long g_trace[8][4096];
     if (more) {                                                 \
       _Pragma("unroll") for (int g_ = 1; g_ < kG; ++g_) LOSA_TL_NEXT((grp)[g_]); \
     }                                                           \
+  } while (0)
+
+// Scheduler side: append n <= 32 entries at once, lane i holding entry i (whole warp).
+#define LOSA_TL_PUT_BULK(ent, n)                                                      \
+  do {                                                                                \
+    const uint32_t first_ = te, last_ = te + (uint32_t)(n) - 1;                       \
+    if ((first_ & 31) == 0)                                                           \
+      LOSA_WAIT_RELAXED(&ctl->tl_empty[(first_ >> 5) & (kTlChunks - 1)],              \
+                        ((first_ / (kTlChunks * 32)) & 1) ^ 1);                       \
+    if ((last_ >> 5) != (first_ >> 5))                                                \
+      LOSA_WAIT_RELAXED(&ctl->tl_empty[(last_ >> 5) & (kTlChunks - 1)],               \
+                        ((last_ / (kTlChunks * 32)) & 1) ^ 1);                        \
+    if (lane < (n)) ctl->tl[(first_ + lane) & (kTlChunks * 32 - 1)] = (ent);          \
+    __syncwarp();                                                                     \
+    if (lane == 0) {                                                                  \
+      if ((last_ >> 5) != (first_ >> 5))                                              \
+        ptx::mbar_arrive(&ctl->tl_full[(first_ >> 5) & (kTlChunks - 1)]);             \
+      if ((last_ & 31) == 31) ptx::mbar_arrive(&ctl->tl_full[(last_ >> 5) & (kTlChunks - 1)]); \
+    }                                                                                 \
+    te += (uint32_t)(n);                                                              \
   } while (0)
 
 // Scheduler side: append one entry (whole warp; lane 0 writes).
@@ -621,20 +550,36 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         w = p.split_first + r / parts;
         flags = kTlPartial | ((uint32_t)part << 24);
       }
+      const int unit = (flags != 0) ? p.split_first + (w - p.split_first) * parts + part : w;
       const int bh = w / p.nPairs, pr = w % p.nPairs;
       LOSA_TL_PUT(kTlItem | flags | (uint32_t)w);
-      TileIter<kNB> it;
-      it.init(p, MODE != kSparse, bh, 2 * pr * kQBT, lane, part, parts);
-      int j, emitted = 0;
-      uint32_t memb;
-      while (it.next(j, memb)) {
-        LOSA_TL_PUT((uint32_t)j | (memb << 16));
-        ++emitted;
+      if (MODE == kSparse) {
+        // the unit's merged tile list was built before the launch: stream it into the ring,
+        // 32 entries per step, so that this warp takes next to no issue slots from the softmax
+        // warps of its scheduler partition
+        const int cnt = __ldg(p.tl_count + unit);
+        const uint32_t* src = p.tl_entries + (int64_t)unit * p.tl_cap;
+        for (int base = 0; base < cnt; base += 32) {
+          const int n = min(32, cnt - base);
+          const uint32_t e = (lane < n) ? __ldg(src + base + lane) : 0u;
+          LOSA_TL_PUT_BULK(e, n);
+        }
+        continue;
       }
-      // K/V tiles are groups of kG entries: pad the item's last group
-      while (emitted % kG != 0) {
-        LOSA_TL_PUT(kTlPad);
-        ++emitted;
+      // dense modes: every key block of the unit's share of the key range, listed by every query
+      // block of the item that exists; K/V tiles are groups of kG entries, the last group is padded
+      uint32_t memb = 0;
+#pragma unroll
+      for (int n = 0; n < kNB; ++n)
+        if (2 * pr * kQBT + n < p.nQb) memb |= 1u << n;
+      const int jlo = (int)(((int64_t)p.nKb * part) / parts);
+      const int jhi = (int)(((int64_t)p.nKb * (part + 1)) / parts);
+      const int cnt = (jhi - jlo + kG - 1) / kG * kG;
+      for (int base = 0; base < cnt; base += 32) {
+        const int n = min(32, cnt - base);
+        const int j = jlo + base + lane;
+        const uint32_t e = (j < jhi) ? ((uint32_t)j | (memb << 16)) : kTlPad;
+        LOSA_TL_PUT_BULK(e, n);
       }
     }
     LOSA_TL_PUT(kTlEnd);
@@ -959,11 +904,90 @@ teardown:
   }
 }
 
+#undef LOSA_TL_PUT_BULK
 #undef LOSA_TL_NEXT_TILE
 #undef LOSA_TL_NEXT
 #undef LOSA_TL_PUT
 #undef LOSA_WAIT_RELAXED
 #undef LOSA_WAIT
+
+// Sparse mode, before the attention kernel: one warp per work unit merges the index lists of the
+// unit's query blocks into its tile list (entry = key block index | membership bits << 16, in
+// ascending order, padded to whole K/V tiles of G entries).  Every list becomes a bitmap in shared
+// memory (coalesced reads, one atomicOr per index), the union's set bits are enumerated 32 words
+// at a time with a warp scan.  Doing this ahead of the launch keeps the in-kernel scheduler warp,
+// which shares a scheduler partition with two softmax warps and is favoured over them, nearly
+// idle.  A unit that is a part of an item takes the same share, by position, of every list, so
+// each (query block, key block) pair belongs to exactly one part.  Indices out of range are
+// reported and skipped; an unsorted list still gives a valid (sorted) tile list.
+template <int NB, int G>
+__global__ void __launch_bounds__(32) build_tile_lists_kernel(const Params p) {
+  extern __shared__ uint32_t bm[];  // [NB][W] bitmaps
+  const int lane = threadIdx.x, unit = blockIdx.x;
+  int w = unit, part = 0, parts = 1;
+  if (unit >= p.split_first) {
+    const int r = unit - p.split_first;
+    parts = p.split_parts;
+    part = r % parts;
+    w = p.split_first + r / parts;
+  }
+  const int bh = w / p.nPairs, pr = w % p.nPairs;
+  const int W = (p.nKb + 31) >> 5;
+  for (int i = lane; i < NB * W; i += 32) bm[i] = 0u;
+  __syncwarp();
+  const int32_t nnz = __ldg(p.offsets + (int64_t)p.B * p.H * p.nQb);
+#pragma unroll
+  for (int n = 0; n < NB; ++n) {
+    const int g = pr * NB + n;
+    if (g >= p.nQb) continue;
+    const int64_t row = (int64_t)bh * p.nQb + g;
+    const int32_t b = __ldg(p.offsets + row), e = __ldg(p.offsets + row + 1);
+    if (b < 0 || e < b || e > nnz || e - b > p.nKb) {
+      report_error(p.status, LOSA_ERR_BAD_INDEX);
+      continue;
+    }
+    const int b2 = b + (int)(((int64_t)(e - b) * part) / parts);
+    const int e2 = b + (int)(((int64_t)(e - b) * (part + 1)) / parts);
+    for (int i = b2 + lane; i < e2; i += 32) {
+      const int v = __ldg(p.kv_idx + i);
+      if ((unsigned)v < (unsigned)p.nKb) atomicOr(&bm[n * W + (v >> 5)], 1u << (v & 31));
+      else report_error(p.status, LOSA_ERR_BAD_INDEX);  // skipped, never used as an address
+    }
+  }
+  __syncwarp();
+  uint32_t* dst = p.tl_entries + (int64_t)unit * p.tl_cap;
+  int cnt = 0;
+  for (int w0 = 0; w0 < W; w0 += 32) {
+    const int wi = w0 + lane;
+    uint32_t m[NB], u = 0;
+#pragma unroll
+    for (int n = 0; n < NB; ++n) {
+      m[n] = (wi < W) ? bm[n * W + wi] : 0u;
+      u |= m[n];
+    }
+    const int c = __popc(u);
+    int incl = c;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += t;
+    }
+    const int total = __shfl_sync(0xffffffffu, incl, 31);
+    uint32_t* out = dst + cnt + (incl - c);
+    while (u) {
+      const int bit = __ffs(u) - 1;
+      u &= u - 1;
+      uint32_t memb = 0;
+#pragma unroll
+      for (int n = 0; n < NB; ++n) memb |= ((m[n] >> bit) & 1u) << n;
+      *out++ = (uint32_t)(wi * 32 + bit) | (memb << 16);
+    }
+    cnt += total;
+  }
+  const int pad = (G - cnt % G) % G;
+  if (lane < pad) dst[cnt + lane] = kTlPad;
+  if (lane == 0) p.tl_count[unit] = cnt + pad;
+}
 
 // Merge of the partial units: for every row of the split items, combine the parts' unnormalised
 // O, reference maximum and row sum (the usual log-sum-exp merge) and write the attention output.
@@ -1132,6 +1156,11 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
     }
   }
   const int grid = min(ctas, prm.nUnits);
+  if (MODE == kSparse) {
+    const size_t bm_bytes = (size_t)C::kNB * ((prm.nKb + 31) / 32) * sizeof(uint32_t);  // <= 32 KB
+    build_tile_lists_kernel<C::kNB, C::kG><<<prm.nUnits, 32, bm_bytes, st>>>(prm);
+    LOSA_CUDA_TRY(cudaGetLastError());
+  }
   kern<<<grid, kThreads, smem, st>>>(mq, mk, mv, prm);
   LOSA_CUDA_TRY(cudaGetLastError());
   if (prm.split_parts > 1) {
@@ -1148,7 +1177,7 @@ int dispatch(const Geometry& g, const void* q, const void* k, const void* v, con
   // sparse forward with 64 x 64 blocks: a 128-row query tile then spans two query blocks and a
   // 128-key tile two key blocks, and with four index lists per work item nearly every tile is
   // visited by somebody while half of its rows sit idle (measured at the CogVideoX shape:
-  // 7.34 ms with 128-key tiles, 6.86 ms with 64-key tiles).
+  // 7.31 ms with 128-key tiles, 6.69 ms with 64-key tiles).
 #define LOSA_CASE(d, r, c)                                                          \
   if (g.D == d && g.R == r && g.C == c)                                             \
   return launch_t<d, r, c, MODE, (r == 64 && c == 64 && MODE == kSparse) ? 64 : 128>(g, q, k, v, prm, st)
@@ -1172,11 +1201,26 @@ extern "C" int losa_debug_trace(void* host, size_t bytes) {
 }
 #endif
 
+namespace {
+size_t part_o_bytes(const Geometry& g) {
+  return (size_t)kMaxPersistentCtas * 2 * 128 * (size_t)g.D * sizeof(float);
+}
+// the last wave's items are cut into at most one unit per CTA
+int64_t max_units(const Geometry& g) { return (int64_t)g.B * g.H * g.nPairs + kMaxPersistentCtas; }
+int tile_list_cap(const Geometry& g) { return (g.nKb + 4 + 31) / 32 * 32; }  // union <= nKb, + padding
+size_t tl_count_bytes(const Geometry& g) { return ((size_t)max_units(g) * sizeof(int32_t) + 255) / 256 * 256; }
+}  // namespace
+
 size_t attn_workspace_bytes(AttnMode mode, const Geometry& g) {
   // attention output: counter, then one slot per partial unit (at most one per CTA) holding the
   // rows' (max, sum) and unnormalised O of both query tiles
-  if (mode == kDense || mode == kSparse)
-    return kCounterBytes + kPartMlBytes + (size_t)kMaxPersistentCtas * 2 * 128 * (size_t)g.D * sizeof(float);
+  if (mode == kDense || mode == kSparse) {
+    size_t bytes = kCounterBytes + kPartMlBytes + part_o_bytes(g);
+    // sparse: the units' merged tile lists (count per unit, then tl_cap entries per unit)
+    if (mode == kSparse)
+      bytes += tl_count_bytes(g) + (size_t)max_units(g) * tile_list_cap(g) * sizeof(uint32_t);
+    return bytes;
+  }
   // counter, per-CTA row statistics, per-CTA table of one entry per row and key tile
   return kCounterBytes + kRowstatBytes +
          (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2);
@@ -1210,6 +1254,12 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
                                         ((mode == kMass || mode == kFused) ? kRowstatBytes : 0));
   prm.part_ml = reinterpret_cast<float2*>(static_cast<char*>(ws) + kCounterBytes);
   prm.part_o = reinterpret_cast<float*>(static_cast<char*>(ws) + kCounterBytes + kPartMlBytes);
+  {
+    char* tl = static_cast<char*>(ws) + kCounterBytes + kPartMlBytes + part_o_bytes(g);
+    prm.tl_count = reinterpret_cast<int32_t*>(tl);
+    prm.tl_entries = reinterpret_cast<uint32_t*>(tl + tl_count_bytes(g));
+    prm.tl_cap = tile_list_cap(g);
+  }
   prm.scale_log2 = g.scale * kLog2e;
   prm.status = status_word_device();
   if (!prm.status) return LOSA_ERR_CUDA;
