@@ -484,9 +484,11 @@ def main():
             "algorithmic_bytes_per_launch": 4 * q0.numel() * 2,
         },
         "clocks": clocks.summary(),
-        # per step: mass 1, select 3, sparse `draws`, dense 1, fused 1; each attention-only call adds
-        # its merge kernel when the last wave of work items is cut into parts
-        "gpu_launches": args.steps * (1 + 3 + (args.draws + 1) * (2 if merge_kernel_runs(wl) else 1) + 1),
+        # per step: mass 1, select 3, `draws` sparse calls of 2 kernels (tile-list pre-pass + attention),
+        # dense 1, fused 1; each attention-only call adds its merge kernel when the last wave of work
+        # items is cut into parts
+        "gpu_launches": args.steps * (1 + 3 + args.draws * (2 + int(merge_kernel_runs(wl)))
+                                      + 1 + int(merge_kernel_runs(wl)) + 1),
     }
     if e2e is not None:
         line["e2e"] = e2e
