@@ -70,6 +70,7 @@ constexpr int kMaxParts = 8;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;
+constexpr float kSafeRowSum = 1.099511627776e12f;  // 2^40: a tile's row sum beyond this re-centres the reference
 
 template <int D, int R, int C_, int MODE, int KT>
 struct Cfg {
@@ -612,6 +613,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const int T = 2 * pr + qt;
       const int grow = T * 128 + row;
       float m_ref = -INFINITY, l = 0.f;
+      bool have_ref = false;  // this warp's rows have a reference maximum (after their first tile)
       uint32_t pv_item = 0;
       float2* tab = nullptr;
       if (C::kWantMass)
@@ -653,94 +655,120 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         TR(3, nsub);
         if (!C::kHasV) {
-          // mass pass: S is in registers, hand the buffer back
+          // mass pass: S is in registers, hand the buffer back (it always computes the maximum, so
+          // there is no second pass that would read S again)
           ptx::tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&ctl->s_free[qt][buf]);
         }
         if (mine) {
-          // Keys that do not exist (>= N) and key blocks the row's query block does not list get
-          // a score of -inf: they drop out of the maximum and their p is exactly 0.  Straight-line
-          // code over all 128 columns is faster than skipping blocks (measured: branches between
-          // the blocks cost the softmax 0.9 k cycles per tile at C = 32).
-          if (!full) {
+          // p = 2^(s * scale_log2 - m_ref) with a reference m_ref that is NOT the running maximum:
+          // the result o = sum(p v) / sum(p) does not depend on it, it only has to keep p inside
+          // the fp32 / bf16 range.  So the common path computes no row maximum at all: it
+          // exponentiates against the reference it has and looks at the tile's row sums; only if a
+          // sum left the safe range (> 2^40, inf or NaN; or there is no reference yet, in the
+          // first tile of an item) does the warp compute the maximum, move the reference, rescale
+          // O and the row sum, and exponentiate the tile again.  P is therefore stored only after
+          // that test (S stays intact in TMEM for the second pass).
+          float2 acc[kG][2];  // row sums per key block (the mass pass needs them apart), two chains each
+          float gsum[kG], tsum = 0.f;
+          // (The mass pass keeps the running maximum: it is bound by the exponentials, its two
+          // warpgroups run side by side, and handing S back early matters more there.)
+          // (All rows of a warp belong to one query block and have seen the same tiles, so
+          // whether a reference exists is known per warp without a vote.)
+          bool recentre = !C::kHasV || !have_ref;
+          have_ref = true;
+#pragma unroll 1
+          for (int pass = 0; pass < 2; ++pass) {
+            // Keys that do not exist (>= N) and key blocks the row's query block does not list
+            // get a score of -inf: their p is exactly 0.  Straight-line code over all 128 columns
+            // is faster than skipping blocks (measured: branches between the blocks cost the
+            // softmax 0.9 k cycles per tile at C = 32).
+            if (!full) {
 #pragma unroll
-            for (int c = 0; c < kW; ++c)
-              if ((c % kC) >= vc[c / kC]) sr[c] = 0xff800000u;
-          }
-          float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
-          float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
+              for (int c = 0; c < kW; ++c)
+                if ((c % kC) >= vc[c / kC]) sr[c] = 0xff800000u;
+            }
+            if (recentre) {
+              float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
+              float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
 #pragma unroll
-          for (int c = 4; c + 8 <= kW; c += 8) {
-            mx0 = ptx::max3(mx0, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
-            mx1 = ptx::max3(mx1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
-            mx2 = ptx::max3(mx2, __uint_as_float(sr[c + 4]), __uint_as_float(sr[c + 5]));
-            mx3 = ptx::max3(mx3, __uint_as_float(sr[c + 6]), __uint_as_float(sr[c + 7]));
-          }
-          mx0 = ptx::max3(mx0, __uint_as_float(sr[kW - 4]), __uint_as_float(sr[kW - 3]));
-          mx1 = ptx::max3(mx1, __uint_as_float(sr[kW - 2]), __uint_as_float(sr[kW - 1]));
-          const float m_new =
-              fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
-          const bool need = m_new > m_ref + kRescaleThreshold;
-          TR(4, nsub);
-          if (__any_sync(0xffffffffu, need)) {
-            const float alpha = need ? ptx::ex2_approx(m_ref - m_new) : 1.f;
-            if (need) m_ref = m_new;
-            l *= alpha;
-            if (C::kHasV && pv_item > 0) {
-              const float2 a2 = make_float2(alpha, alpha);
+              for (int c = 4; c + 8 <= kW; c += 8) {
+                mx0 = ptx::max3(mx0, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
+                mx1 = ptx::max3(mx1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
+                mx2 = ptx::max3(mx2, __uint_as_float(sr[c + 4]), __uint_as_float(sr[c + 5]));
+                mx3 = ptx::max3(mx3, __uint_as_float(sr[c + 6]), __uint_as_float(sr[c + 7]));
+              }
+              mx0 = ptx::max3(mx0, __uint_as_float(sr[kW - 4]), __uint_as_float(sr[kW - 3]));
+              mx1 = ptx::max3(mx1, __uint_as_float(sr[kW - 2]), __uint_as_float(sr[kW - 1]));
+              const float m_new =
+                  fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
+              // rows whose reference is close enough keep it
+              const bool need = m_new > m_ref + kRescaleThreshold;
+              const float alpha = need ? ptx::ex2_approx(m_ref - m_new) : 1.f;
+              if (need) m_ref = m_new;
+              l *= alpha;
+              if (C::kHasV && pv_item > 0) {
+                // (every earlier product into O is complete: s_full covers them)
+                const float2 a2 = make_float2(alpha, alpha);
 #pragma unroll
-              for (int c0 = 0; c0 < D; c0 += 32) {
-                uint32_t r[32];
-                ptx::tmem_ld32(tO + c0, r);
-                ptx::tmem_wait_ld();
+                for (int c0 = 0; c0 < D; c0 += 32) {
+                  uint32_t r[32];
+                  ptx::tmem_ld32(tO + c0, r);
+                  ptx::tmem_wait_ld();
 #pragma unroll
-                for (int c = 0; c < 32; c += 2) {
-                  const float2 v = ptx::mul2(
-                      make_float2(__uint_as_float(r[c]), __uint_as_float(r[c + 1])), a2);
-                  r[c] = __float_as_uint(v.x);
-                  r[c + 1] = __float_as_uint(v.y);
+                  for (int c = 0; c < 32; c += 2) {
+                    const float2 v = ptx::mul2(
+                        make_float2(__uint_as_float(r[c]), __uint_as_float(r[c + 1])), a2);
+                    r[c] = __float_as_uint(v.x);
+                    r[c + 1] = __float_as_uint(v.y);
+                  }
+                  ptx::tmem_st32(tO + c0, r);
                 }
-                ptx::tmem_st32(tO + c0, r);
               }
             }
-          }
-          // p = 2^(s * scale_log2 - m_ref), two columns per instruction; the bf16 pairs
-          // overwrite the low half of the register array
-          TR(5, nsub);
-          const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
-          const float2 nm2 = make_float2(-m_ref, -m_ref);
-          // (row sums per key block: the mass pass needs them apart; two chains per block)
-          float2 acc[kG][2];
+            TR(5, nsub);
+            // two columns per instruction; the bf16 pairs overwrite the low half of the registers
+            const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+            const float2 nm2 = make_float2(-m_ref, -m_ref);
 #pragma unroll
-          for (int g = 0; g < kG; ++g) acc[g][0] = acc[g][1] = make_float2(0.f, 0.f);
+            for (int g = 0; g < kG; ++g) acc[g][0] = acc[g][1] = make_float2(0.f, 0.f);
 #pragma unroll
-          for (int c = 0; c < kW; c += 4) {
-            float2 x0 = ptx::fma2(
-                make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2);
-            float2 x1 = ptx::fma2(
-                make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, nm2);
-            x0.x = ptx::ex2_approx(x0.x);
-            x0.y = ptx::ex2_approx(x0.y);
-            x1.x = ptx::ex2_approx(x1.x);
-            x1.y = ptx::ex2_approx(x1.y);
-            acc[c / kC][0] = ptx::add2(acc[c / kC][0], x0);
-            acc[c / kC][1] = ptx::add2(acc[c / kC][1], x1);
-            if (C::kHasV) {
-              sr[c >> 1] = ptx::pack_bf16x2(x0.x, x0.y);
-              sr[(c >> 1) + 1] = ptx::pack_bf16x2(x1.x, x1.y);
-              // 64 keys of P are complete: store them while the rest is computed
-              if ((c & 63) == 60) ptx::tmem_st32(tSb + (c >> 6) * 32, &sr[(c >> 6) * 32]);
+            for (int c = 0; c < kW; c += 4) {
+              float2 x0 = ptx::fma2(
+                  make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2);
+              float2 x1 = ptx::fma2(
+                  make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, nm2);
+              x0.x = ptx::ex2_approx(x0.x);
+              x0.y = ptx::ex2_approx(x0.y);
+              x1.x = ptx::ex2_approx(x1.x);
+              x1.y = ptx::ex2_approx(x1.y);
+              acc[c / kC][0] = ptx::add2(acc[c / kC][0], x0);
+              acc[c / kC][1] = ptx::add2(acc[c / kC][1], x1);
+              if (C::kHasV) {
+                sr[c >> 1] = ptx::pack_bf16x2(x0.x, x0.y);
+                sr[(c >> 1) + 1] = ptx::pack_bf16x2(x1.x, x1.y);
+              }
             }
-          }
-          TR(6, nsub);
-          float gsum[kG], tsum = 0.f;
+            TR(6, nsub);
+            tsum = 0.f;
 #pragma unroll
-          for (int g = 0; g < kG; ++g) {
-            gsum[g] = (acc[g][0].x + acc[g][0].y) + (acc[g][1].x + acc[g][1].y);
-            tsum += gsum[g];
+            for (int g = 0; g < kG; ++g) {
+              gsum[g] = (acc[g][0].x + acc[g][0].y) + (acc[g][1].x + acc[g][1].y);
+              tsum += gsum[g];
+            }
+            // after a pass with a fresh maximum every p is at most 2^8
+            if (recentre || !__any_sync(0xffffffffu, !(tsum <= kSafeRowSum))) break;
+            recentre = true;
+#pragma unroll
+            for (int c0 = 0; c0 < kW; c0 += 32) ptx::tmem_ld32(tSb + c0, &sr[c0]);
+            ptx::tmem_wait_ld();
           }
           l += tsum;
+          if (C::kHasV) {
+#pragma unroll
+            for (int c0 = 0; c0 < kW / 2; c0 += 32) ptx::tmem_st32(tSb + c0, &sr[c0]);
+          }
           if (C::kWantMass) {
             // one table entry per key block
 #pragma unroll

@@ -115,8 +115,9 @@ def test_fused_construction_step_matches_oracle_and_the_separate_calls(shape):
     qn, kn, vn = util.to_np(q), util.to_np(k), util.to_np(v)
     util.assert_output_close(o, orc.dense_attn(qn, kn, vn), f"fused o {shape}")
     # same tiles and arithmetic; the separate call may cut its last work items into parts of the key
-    # range and merge them, which changes the summation order, not the result beyond rounding
-    assert (o - o_sep).abs().max().item() <= util.MAX_ABS_TOL
+    # range and merge them, which changes the summation order, not the result beyond rounding: two
+    # approximations, each within the tolerance of the exact result
+    assert (o - o_sep).abs().max().item() <= 2 * util.MAX_ABS_TOL
     ref, ref_lse = orc.block_mass(qn, kn, BLK, BLK, return_lse=True)
     got = mass.cpu().numpy().reshape(ref.shape).astype(np.float64)
     assert np.abs(got - ref).max() <= util.MASS_TOL

@@ -121,9 +121,9 @@ def test_full_size_parity_on_sampled_query_blocks(name, n_sample):
         o_f, mass_f = losa.losa_attn_mass(qd, kd, vd, wl.R, wl.C, out_dtype=torch.float32)
         o_d = losa.losa_attn(qd, kd, vd, wl.R, wl.C, out_dtype=torch.float32)
         losa.check_async("fused construction")
-        # the attention-only call cuts its last work items into parts and merges them: same result up
-        # to the summation order
-        assert (o_f - o_d).abs().max().item() <= util.MAX_ABS_TOL
+        # two approximations of the same values (the attention-only call also cuts its last work items
+        # into parts and merges them): each is within the tolerance of the exact result
+        assert (o_f - o_d).abs().max().item() <= 2 * util.MAX_ABS_TOL
         gmf = mass_f.cpu().numpy().reshape(wl.rows, wl.nKb)
         assert float(np.abs(gmf[ids] - ref_mass).max()) <= util.MASS_TOL
         assert np.abs(gmf.astype(np.float64).sum(1) - 1.0).max() <= util.MASS_TOL
