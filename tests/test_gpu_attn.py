@@ -352,3 +352,43 @@ def test_rectangular_blocks_match_oracle(shape):
         ref_o = orc.blocks_to_tokens(orc.sparse_attn(qn, kn, vn, R, C, o_h.astype(np.int32),
                                                      i_h.astype(np.int32)), B, H, N)
         util.assert_output_close(o_s, ref_o, f"sparse {name} {shape}")
+
+
+@pytest.mark.parametrize("D,BLK", [(128, 128), (64, 64), (64, 128)])
+@pytest.mark.parametrize("jump", [6.0, 35.0, 110.0])
+def test_scores_that_jump_far_above_the_first_tiles(D, BLK, jump):
+    """The attention kernels exponentiate against a reference that only moves when a tile's row sums
+    leave the safe range.  Scores that rise by `jump` nats after the first key tiles (p would reach
+    2^(jump * 1.44): within range, beyond 2^40, beyond fp32) must give the exact softmax all the
+    same, for dense and sparse attention and for the fused pass."""
+    losa = lib()
+    B, H, N = 1, 2, 128 * 5 + 40
+    g = torch.Generator("cpu").manual_seed(5)
+    q = torch.randn(B, H, N, D, generator=g) * 0.3 + 1.0   # q . ones(D) is about D
+    k = torch.randn(B, H, N, D, generator=g) * 0.3
+    # keys from 256 on: an added component along ones(D) that lifts q.k / sqrt(D) by about `jump`,
+    # rising in two steps (at 256 and at 448) so that the reference has to move more than once
+    lift = jump * (D ** 0.5) / D
+    k[:, :, 256:] += 0.5 * lift
+    k[:, :, 448:] += 0.5 * lift
+    v = torch.randn(B, H, N, D, generator=g)
+    q, k, v = q.bfloat16(), k.bfloat16(), v.bfloat16()
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    qn, kn, vn = util.to_np(q), util.to_np(k), util.to_np(v)
+    ref = orc.dense_attn(qn, kn, vn)
+    o = losa.losa_attn(qd, kd, vd, BLK, BLK, out_dtype=torch.float32)
+    assert losa.losa_async_status() == 0
+    assert torch.isfinite(o).all()
+    util.assert_output_close(o, ref, f"dense jump {jump}")
+    o_f, mass = losa.losa_attn_mass(qd, kd, vd, BLK, BLK, out_dtype=torch.float32)
+    assert losa.losa_async_status() == 0
+    util.assert_output_close(o_f, ref, f"fused jump {jump}")
+    ref_m = orc.block_mass(qn, kn, BLK, BLK)
+    assert np.abs(mass.cpu().numpy().reshape(ref_m.shape) - ref_m).max() <= util.MASS_TOL
+    nb = -(-N // BLK)
+    off, idx = util.random_csr(B * H * nb, nb, 3, 0.6)
+    o_s = losa.losa_sparse_attn(qd, kd, vd, torch.from_numpy(off).cuda(), torch.from_numpy(idx).cuda(),
+                                BLK, BLK, out_dtype=torch.float32)
+    assert losa.losa_async_status() == 0
+    ref_s = orc.blocks_to_tokens(orc.sparse_attn(qn, kn, vn, BLK, BLK, off, idx), B, H, N)
+    util.assert_output_close(o_s, ref_s, f"sparse jump {jump}")
