@@ -630,7 +630,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // the row's query block lists the block, none otherwise (nor for a padding entry)
         uint32_t memb = 0;
         int vc[kG];
-        bool mine = false, full = true;
+        bool mine = false, full = true, ragged = false;
 #pragma unroll
         for (int g = 0; g < kG; ++g) {
           memb |= (grp[g] >> 16) & 0xfu;
@@ -638,6 +638,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           vc[g] = ((grp[g] >> (16 + my_bit)) & 1u) ? min(kC, p.N - jg * kC) : 0;
           mine = mine || vc[g] > 0;
           full = full && vc[g] == kC;
+          ragged = ragged || (vc[g] > 0 && vc[g] < kC);  // the sequence's last, short key block
         }
         if (((memb >> (qt * kQBT)) & kQMask) == 0) continue;
         const uint32_t buf = nsub % kNS;
@@ -680,11 +681,13 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           have_ref = true;
 #pragma unroll 1
           for (int pass = 0; pass < 2; ++pass) {
-            // Keys that do not exist (>= N) and key blocks the row's query block does not list
-            // get a score of -inf: their p is exactly 0.  Straight-line code over all 128 columns
-            // is faster than skipping blocks (measured: branches between the blocks cost the
-            // softmax 0.9 k cycles per tile at C = 32).
-            if (!full) {
+            // Key blocks the row's query block does not list must give p = 0: on the common path
+            // that costs nothing, their columns simply get -inf instead of -m_ref as the addend
+            // of the scaling FMA (straight-line code over all 128 columns; skipping blocks with
+            // branches was measured 0.9 k cycles per tile slower at C = 32).  Scores are set to
+            // -inf column by column only where single keys do not exist (>= N, in the sequence's
+            // last key block) and on the re-centring pass, whose maximum must not see them.
+            if (ragged || (recentre && !full)) {
 #pragma unroll
               for (int c = 0; c < kW; ++c)
                 if ((c % kC) >= vc[c / kC]) sr[c] = 0xff800000u;
@@ -730,15 +733,19 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             TR(5, nsub);
             // two columns per instruction; the bf16 pairs overwrite the low half of the registers
             const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
-            const float2 nm2 = make_float2(-m_ref, -m_ref);
+            float2 nm2[kG];
 #pragma unroll
-            for (int g = 0; g < kG; ++g) acc[g][0] = acc[g][1] = make_float2(0.f, 0.f);
+            for (int g = 0; g < kG; ++g) {
+              const float a = (vc[g] > 0) ? -m_ref : -INFINITY;
+              nm2[g] = make_float2(a, a);
+              acc[g][0] = acc[g][1] = make_float2(0.f, 0.f);
+            }
 #pragma unroll
             for (int c = 0; c < kW; c += 4) {
               float2 x0 = ptx::fma2(
-                  make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2);
+                  make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2[c / kC]);
               float2 x1 = ptx::fma2(
-                  make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, nm2);
+                  make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, nm2[c / kC]);
               x0.x = ptx::ex2_approx(x0.x);
               x0.y = ptx::ex2_approx(x0.y);
               x1.x = ptx::ex2_approx(x1.x);
@@ -1201,14 +1208,9 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
 template <int MODE>
 int dispatch(const Geometry& g, const void* q, const void* k, const void* v, const Params& prm,
              cudaStream_t st) {
-  // K/V tiles of 128 keys (128 / C gathered key blocks, 128-wide MMAs) everywhere but in the
-  // sparse forward with 64 x 64 blocks: a 128-row query tile then spans two query blocks and a
-  // 128-key tile two key blocks, and with four index lists per work item nearly every tile is
-  // visited by somebody while half of its rows sit idle (measured at the CogVideoX shape:
-  // 7.31 ms with 128-key tiles, 6.69 ms with 64-key tiles).
-#define LOSA_CASE(d, r, c)                                                          \
-  if (g.D == d && g.R == r && g.C == c)                                             \
-  return launch_t<d, r, c, MODE, (r == 64 && c == 64 && MODE == kSparse) ? 64 : 128>(g, q, k, v, prm, st)
+  // K/V tiles of 128 keys everywhere (128 / C gathered key blocks, 128-wide MMAs)
+#define LOSA_CASE(d, r, c) \
+  if (g.D == d && g.R == r && g.C == c) return launch_t<d, r, c, MODE, 128>(g, q, k, v, prm, st)
   LOSA_CASE(128, 128, 128);
   LOSA_CASE(64, 64, 64);
   LOSA_CASE(128, 128, 32);  // the paper's own block geometry

@@ -79,11 +79,7 @@ def test_sparse_with_all_blocks_equals_own_dense(shape):
                                 BLK, BLK, out_dtype=torch.float32)
     o_d = losa.losa_attn(q, k, v, BLK, BLK, out_dtype=torch.float32)
     assert losa.losa_async_status() == 0
-    if BLK == 128:
-        assert torch.equal(o_s, o_d)  # same tiles in the same order: bit-identical
-    else:
-        # 64 x 64 blocks: the sparse forward walks 64-key tiles, the dense one 128-key tiles
-        assert (o_s - o_d).abs().max().item() <= util.MAX_ABS_TOL
+    assert torch.equal(o_s, o_d)  # same tiles in the same order: bit-identical
 
 
 @pytest.mark.parametrize("shape", SHAPES)
