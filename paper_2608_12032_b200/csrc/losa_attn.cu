@@ -245,6 +245,12 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   constexpr int kC = C::kC, kG = C::kG, kQBT = C::kQBT, kNB = C::kNB, kW = C::kW, kNS = C::kNS;
   constexpr uint32_t kSStride = C::kSStride, kNVs = C::kNV > 0 ? C::kNV : 1;
   constexpr uint32_t kQMask = (1u << kQBT) - 1u;
+  // The mass pass is bound by the special-function unit (16 exponentials per clock and SM): every
+  // fourth group of four exponentials computes two of them with a polynomial on the FMA pipe
+  // instead (12.5 % of all; measured 4.92 -> 4.63 ms at the Wan shape; a quarter or half of them
+  // is slower, 5.6 and 5.8 ms: the loop turns issue-bound).  Not in the attention modes, which
+  // wait on the chain of their steps, not on that unit (tried twice, slower each time).
+  constexpr int kPolyEvery = (MODE == kMass) ? 4 : 0;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -748,8 +754,12 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                   make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, nm2[c / kC]);
               x0.x = ptx::ex2_approx(x0.x);
               x0.y = ptx::ex2_approx(x0.y);
-              x1.x = ptx::ex2_approx(x1.x);
-              x1.y = ptx::ex2_approx(x1.y);
+              if (kPolyEvery > 0 && ((c >> 2) % (kPolyEvery > 0 ? kPolyEvery : 1)) == 0) {
+                x1 = ptx::ex2_poly2(x1);  // mass pass: a share of the exponentials on the FMA pipe
+              } else {
+                x1.x = ptx::ex2_approx(x1.x);
+                x1.y = ptx::ex2_approx(x1.y);
+              }
               acc[c / kC][0] = ptx::add2(acc[c / kC][0], x0);
               acc[c / kC][1] = ptx::add2(acc[c / kC][1], x1);
               if (C::kHasV) {
