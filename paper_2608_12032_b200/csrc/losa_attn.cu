@@ -2,35 +2,34 @@
 // frozen CSR pattern (Eq. 4) and the exact block-mass pass (Eq. 1), as ONE warp-specialised
 // persistent kernel template.
 //
-// CTA = 12 warps.  Warps 0-3 are utility warps: warp 0 (one elected thread) is the TMA producer,
-// which streams the query tiles and the K / V tiles named by the block indices into
-// 128B-swizzled shared-memory rings; warps 1 and 2 (one elected thread each) issue the tcgen05
-// MMAs of query tile 0 and 1: S = Q K^T from shared memory into TMEM, O += P V with P read from
-// TMEM (bf16, written over S) and V from shared memory as the MN-major operand; warp 3 walks
-// the block-index lists and publishes the tile list every other warp follows.  Warps 4-7 and
-// 8-11 are two softmax warpgroups, each owning one 128-row query tile (thread = query row =
-// TMEM lane); they take their registers from the utility warpgroup (setmaxnreg).
+// CTA = 12 warps.  Warps 0-3 are utility warps: warp 0 is the TMA producer, which streams the
+// query tiles and the K / V tiles named by the tile list into 128B-swizzled shared-memory rings
+// (a K/V tile is 128 keys: 128 / C key blocks, one copy per block and 64-column slab); warps 1
+// and 2 (one elected thread each) issue the tcgen05 MMAs of query tile 0 and 1: S = Q K^T from
+// shared memory into TMEM, O += P V with P read from TMEM (bf16, written over S) and V from
+// shared memory as the MN-major operand; warp 3 publishes the tile list every other warp
+// follows (sparse mode: streamed from lists that build_tile_lists_kernel made before the
+// launch).  Warps 4-7 and 8-11 are two softmax warpgroups, each owning one 128-row query tile
+// (thread = query row = TMEM lane); they take their registers from the utility warpgroup.
 //
 // A work item is a pair of consecutive query tiles of one (batch, head).  The key blocks the
-// pair visits are the ascending merge of the tiles' index lists (one list per query block;
-// two per tile when the block size is 64), so a K/V tile needed by both is loaded once, and
-// MMAs are issued only for the query tiles that list it.  Query-block rows that do not list
-// a tile of their 128-row group get P = 0 for it.
+// pair visits are the ascending union of the index lists of its query blocks (two lists, four
+// when R = 64), so a K/V tile needed by both tiles is loaded once, and MMAs are issued only for
+// the query tiles that list one of its blocks.  The items of the last, partly filled wave of
+// the persistent grid are cut into parts of their lists, merged by merge_parts_kernel.
 //
-// One S = Q K^T covers a whole key tile (for 128-key tiles, 128-wide MMAs: an MMA costs its
-// issuing thread ~70 cycles whatever its width, so wide MMAs are what keeps the issuer off the
-// critical path).  TMEM then holds exactly S and O of both query tiles, P overwrites S, and
-// per query tile the steps S -> softmax -> O += P V -> next S form a serial chain.  The two
-// tiles run that chain half a period apart: one tile's MMAs execute while the other tile's
-// softmax runs.  Running maxima are updated lazily: O and the row sum are rescaled only when
-// the maximum grew by more than 2^8, which keeps the correction off the common path without
-// losing accuracy (the stale reference bounds p by 2^8).
+// One S = Q K^T covers a whole K/V tile (128-wide MMAs: an MMA costs its issuing thread ~70
+// cycles whatever its width, so wide MMAs are what keeps the issuer off the critical path).
+// TMEM then holds exactly S and O of both query tiles, P overwrites S, and per query tile the
+// steps S -> softmax -> O += P V -> next S form a serial chain.  The two tiles run that chain
+// half a period apart: one tile's MMAs execute while the other tile's softmax runs.  The
+// attention modes keep no running maximum: they exponentiate against a reference that moves
+// only when a tile's row sums leave the safe range (the result does not depend on it).
 //
 // Every wait is bounded; a wait that expires raises the CTA's abort flag, records
 // LOSA_ERR_TIMEOUT, and all roles leave through the common teardown that frees TMEM.
 #include <cuda.h>
 #include <cuda_bf16.h>
-#include <limits.h>
 #include <math.h>
 
 #include "losa_common.cuh"
