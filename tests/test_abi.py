@@ -37,5 +37,19 @@ def test_workspace_sizing_and_status_strings_need_no_gpu():
     assert 0 < binding.losa_workspace_bytes(binding.LOSA_OP_ATTN, p) <= 32 << 20
     bad = binding.Problem(1, 1, 128, 96, 128, 128, 128 * 96, 128 * 96, 96, 0.0)
     assert binding.losa_workspace_bytes(binding.LOSA_OP_BLOCK_MASS, bad) == 0
+    # block geometries: query blocks of 128 rows go with key blocks of 128, 64 or 32 (the paper's own),
+    # query blocks of 64 rows with key blocks of 64 only
+    for R, C, ok in [(128, 128, True), (128, 64, True), (128, 32, True), (64, 64, True), (64, 32, False),
+                     (32, 32, False), (128, 16, False), (64, 128, False)]:
+        g = binding.Problem(1, 2, 1000, 128, R, C, 2 * 1000 * 128, 1000 * 128, 128, 0.0)
+        for op in (binding.LOSA_OP_BLOCK_MASS, binding.LOSA_OP_SPARSE_ATTN, binding.LOSA_OP_ATTN,
+                   binding.LOSA_OP_ATTN_MASS):
+            assert (binding.losa_workspace_bytes(op, g) > 0) == ok, (R, C, op)
+    # the sparse forward also holds the merged tile lists of all work units: grows with N / C
+    small = binding.Problem(1, 12, 32760, 128, 128, 128, 12 * 32760 * 128, 32760 * 128, 128, 0.0)
+    fine = binding.Problem(1, 12, 32760, 128, 128, 32, 12 * 32760 * 128, 32760 * 128, 128, 0.0)
+    assert (binding.losa_workspace_bytes(binding.LOSA_OP_SPARSE_ATTN, fine)
+            > binding.losa_workspace_bytes(binding.LOSA_OP_SPARSE_ATTN, small)
+            > binding.losa_workspace_bytes(binding.LOSA_OP_ATTN, small))
     assert binding.losa_status_string(0) == "LOSA_OK"
     assert binding.losa_status_string(-6) == "LOSA_ERR_TIMEOUT"
