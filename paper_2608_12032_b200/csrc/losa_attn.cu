@@ -956,14 +956,14 @@ teardown:
 #undef LOSA_WAIT
 
 // Sparse mode, before the attention kernel: one warp per work unit merges the index lists of the
-// unit's query blocks into its tile list (entry = key block index | membership bits << 16, in
-// ascending order, padded to whole K/V tiles of G entries).  Every list becomes a bitmap in shared
+// unit's query blocks into its tile list (entry = key block index | membership bits << 16,
+// padded to whole K/V tiles of G entries; for the order see below).  Every list becomes a bitmap in shared
 // memory (coalesced reads, one atomicOr per index), the union's set bits are enumerated 32 words
 // at a time with a warp scan.  Doing this ahead of the launch keeps the in-kernel scheduler warp,
 // which shares a scheduler partition with two softmax warps and is favoured over them, nearly
 // idle.  A unit that is a part of an item takes the same share, by position, of every list, so
 // each (query block, key block) pair belongs to exactly one part.  Indices out of range are
-// reported and skipped; an unsorted list still gives a valid (sorted) tile list.
+// reported and skipped; an unsorted list still gives a valid tile list.
 template <int NB, int G>
 __global__ void __launch_bounds__(32) build_tile_lists_kernel(const Params p) {
   extern __shared__ uint32_t bm[];  // [NB][W] bitmaps
@@ -999,38 +999,89 @@ __global__ void __launch_bounds__(32) build_tile_lists_kernel(const Params p) {
     }
   }
   __syncwarp();
+  // Order of the entries.  A key block that only ONE of the unit's two query tiles lists is
+  // processed by that tile alone, at half the CTA's rate; two such blocks, one of each tile, can
+  // be in flight at the same time (the tiles' chains are independent).  So the list holds first
+  // the blocks both tiles list, then the single-tile blocks of tile 0 and tile 1 in alternation
+  // (K/V tile by K/V tile; a class that does not fill its last K/V tile pads it), then what is
+  // left of the longer class.  Within a class the blocks ascend.  Correctness does not depend on
+  // the order of the key blocks.
   uint32_t* dst = p.tl_entries + (int64_t)unit * p.tl_cap;
-  int cnt = 0;
+  constexpr uint32_t kMaskA = (1u << (NB / 2)) - 1u;
+  int nb = 0, na = 0, nbb = 0;  // both, tile 0 only, tile 1 only
   for (int w0 = 0; w0 < W; w0 += 32) {
     const int wi = w0 + lane;
-    uint32_t m[NB], u = 0;
+    uint32_t ta = 0, tb = 0;
+#pragma unroll
+    for (int n = 0; n < NB; ++n) {
+      const uint32_t m = (wi < W) ? bm[n * W + wi] : 0u;
+      if (n < NB / 2) ta |= m; else tb |= m;
+    }
+    nb += __popc(ta & tb);
+    na += __popc(ta & ~tb);
+    nbb += __popc(tb & ~ta);
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    nb += __shfl_xor_sync(0xffffffffu, nb, d);
+    na += __shfl_xor_sync(0xffffffffu, na, d);
+    nbb += __shfl_xor_sync(0xffffffffu, nbb, d);
+  }
+  const int s1 = (nb + G - 1) / G * G;                       // entries of the first section
+  const int tA = (na + G - 1) / G, tB = (nbb + G - 1) / G;   // K/V tiles of the single-tile classes
+  const int tmin = min(tA, tB);
+  const int total = min(s1 + (tA + tB) * G, p.tl_cap);
+  for (int i = lane; i < total; i += 32) dst[i] = kTlPad;
+  __syncwarp();
+  int rb = 0, ra = 0, rbb = 0;  // entries of each class emitted by earlier windows
+  for (int w0 = 0; w0 < W; w0 += 32) {
+    const int wi = w0 + lane;
+    uint32_t m[NB], ta = 0, tb = 0;
 #pragma unroll
     for (int n = 0; n < NB; ++n) {
       m[n] = (wi < W) ? bm[n * W + wi] : 0u;
-      u |= m[n];
+      if (n < NB / 2) ta |= m[n]; else tb |= m[n];
     }
-    const int c = __popc(u);
-    int incl = c;
+    uint32_t cls[3] = {ta & tb, ta & ~tb, tb & ~ta};
+    int incl[3], tot[3];
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const int t = __shfl_up_sync(0xffffffffu, incl, d);
-      if (lane >= d) incl += t;
-    }
-    const int total = __shfl_sync(0xffffffffu, incl, 31);
-    uint32_t* out = dst + cnt + (incl - c);
-    while (u) {
-      const int bit = __ffs(u) - 1;
-      u &= u - 1;
-      uint32_t memb = 0;
+    for (int k = 0; k < 3; ++k) {
+      incl[k] = __popc(cls[k]);
 #pragma unroll
-      for (int n = 0; n < NB; ++n) memb |= ((m[n] >> bit) & 1u) << n;
-      *out++ = (uint32_t)(wi * 32 + bit) | (memb << 16);
+      for (int d = 1; d < 32; d <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl[k], d);
+        if (lane >= d) incl[k] += t;
+      }
+      tot[k] = __shfl_sync(0xffffffffu, incl[k], 31);
     }
-    cnt += total;
+    const int base[3] = {rb, ra, rbb};
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+      uint32_t u = cls[k];
+      int r = base[k] + incl[k] - __popc(u);  // rank of this lane's first entry within its class
+      while (u) {
+        const int bit = __ffs(u) - 1;
+        u &= u - 1;
+        uint32_t memb = 0;
+#pragma unroll
+        for (int n = 0; n < NB; ++n) memb |= ((m[n] >> bit) & 1u) << n;
+        int pos;
+        if (k == 0) {
+          pos = r;
+        } else {
+          const int t = r / G;  // K/V tile of the class
+          const int slot = (t < tmin) ? 2 * t + (k - 1) : 2 * tmin + (t - tmin);
+          pos = s1 + slot * G + r % G;
+        }
+        if (pos < p.tl_cap) dst[pos] = (uint32_t)(wi * 32 + bit) | (memb << 16);
+        ++r;
+      }
+    }
+    rb += tot[0];
+    ra += tot[1];
+    rbb += tot[2];
   }
-  const int pad = (G - cnt % G) % G;
-  if (lane < pad) dst[cnt + lane] = kTlPad;
-  if (lane == 0) p.tl_count[unit] = cnt + pad;
+  if (lane == 0) p.tl_count[unit] = total;
 }
 
 // Merge of the partial units: for every row of the split items, combine the parts' unnormalised
@@ -1246,7 +1297,7 @@ size_t part_o_bytes(const Geometry& g) {
 }
 // the last wave's items are cut into at most one unit per CTA
 int64_t max_units(const Geometry& g) { return (int64_t)g.B * g.H * g.nPairs + kMaxPersistentCtas; }
-int tile_list_cap(const Geometry& g) { return (g.nKb + 4 + 31) / 32 * 32; }  // union <= nKb, + padding
+int tile_list_cap(const Geometry& g) { return (g.nKb + 16 + 31) / 32 * 32; }  // union <= nKb, + padding of three sections
 size_t tl_count_bytes(const Geometry& g) { return ((size_t)max_units(g) * sizeof(int32_t) + 255) / 256 * 256; }
 }  // namespace
 
