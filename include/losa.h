@@ -56,7 +56,7 @@ enum {
   LOSA_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed                            */
   LOSA_ERR_TIMEOUT = -6,     /* a bounded device-side wait expired (device-side)             */
   LOSA_ERR_BAD_INDEX = -7,   /* kv_idx / offsets out of range or not ascending (device-side) */
-  LOSA_ERR_BAD_MASS = -8     /* negative or NaN mass seen by losa_select (device-side)       */
+  LOSA_ERR_BAD_MASS = -8     /* negative, NaN or > 8 mass seen by losa_select (device-side)  */
 };
 
 enum {

@@ -1,10 +1,14 @@
 // losa_select: retained-mass selection (Eq. 3) and CSR validation.
 //
 // Three small launches over a [rows, nKb] fp32 mass matrix:
-//   1. select_rows_kernel   one CTA per row: sort (mass descending, index ascending) as
-//                           64-bit integer keys in shared memory, fp64 prefix sum along the
-//                           sorted order, shortest prefix reaching tau; the kept set is
-//                           written as a bitmap over block indices plus its size.
+//   1. select_rows_warp_kernel  rows of at most 1024 blocks: one warp per row, the row in
+//                           registers, the threshold value found bit by bit with masked
+//                           fixed-point sums (no sort); the kept set is written as a bitmap
+//                           over block indices plus its size.
+//      select_rows_kernel   longer rows (and the no-allocation entry point): one CTA per
+//                           row, sort (mass descending, index ascending) as 64-bit integer
+//                           keys in shared memory, fp64 prefix sum along the sorted order,
+//                           shortest prefix reaching tau; same outputs.
 //   2. scan_counts_kernel   exclusive prefix of the per-row sizes -> offsets.
 //   3. expand_rows_kernel   one warp per row: bitmap -> ascending block indices.
 // Each mass element is read once and each kept index written once; the bitmap adds 1/16
@@ -113,6 +117,111 @@ select_rows_kernel(const float* __restrict__ mass, int nKb, int n2, double tau, 
   __syncthreads();
   for (int w = tid; w < words; w += kSelThreads) bitmaps[row * words + w] = bitmap[w];
   if (tid == 0) counts[row] = s;
+}
+
+// Rows of at most 1024 blocks: one WARP per row, no sort.  The kept set of Eq. 3 is "every block
+// heavier than v*, plus the lowest-indexed blocks equal to v* until the sum reaches tau", where v*
+// is the largest value v with sum(mass >= v) >= tau.  Non-negative floats order like their bit
+// patterns, so v* is found bit by bit (31 steps), each step one masked sum over the row, which
+// the warp holds in registers (lane l owns blocks l, l + 32, ...).  The sums are taken in 2^-60
+// fixed point: integer addition is exact and order-independent, so the result is deterministic
+// and differs from a sequential fp64 sum by less than 1e-15 (masses below 2^-37 lose low bits).
+// The kept set comes out as one ballot per 32 blocks - the bitmap word - and its size.
+template <int K>  // blocks per lane
+__global__ void __launch_bounds__(128)
+select_rows_warp_kernel(const float* __restrict__ mass, int rows, int nKb, double tau, int fixed_count,
+                        int32_t* __restrict__ counts, uint32_t* __restrict__ bitmaps, int* status) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const int words = (nKb + 31) >> 5;
+  const float* mrow = mass + row * nKb;
+  uint32_t bits[K];
+  unsigned long long fx[K];
+  bool bad = false;
+#pragma unroll
+  for (int k = 0; k < K; ++k) {
+    const int i = k * 32 + lane;
+    float m = (i < nKb) ? mrow[i] : 0.0f;
+    if (!(m >= 0.0f) || m > 8.0f) {  // negative, NaN, or far beyond any mass
+      bad = true;
+      m = 0.0f;
+    }
+    bits[k] = (m == 0.0f) ? 0u : __float_as_uint(m);  // -0 becomes +0
+    // the weight that is summed: the mass in 2^-60 fixed point (exact product), or 1 per existing
+    // block for the fixed-ratio rule, which counts; blocks past the row's end weigh nothing
+    if (fixed_count > 0) fx[k] = (i < nKb) ? 1ull : 0ull;
+    else fx[k] = (unsigned long long)((double)m * 1152921504606846976.0);
+  }
+  if (__any_sync(0xffffffffu, bad) && lane == 0) report_error(status, LOSA_ERR_BAD_MASS);
+
+  // sum (or count, for the fixed-ratio rule) of the blocks with bits >= v, over the whole row
+  auto measure_ge = [&](uint32_t v) -> unsigned long long {
+    unsigned long long a0 = 0ull, a1 = 0ull;
+#pragma unroll
+    for (int k = 0; k < K; k += 2) {
+      a0 += (bits[k] >= v) ? fx[k] : 0ull;
+      a1 += (bits[k + 1] >= v) ? fx[k + 1] : 0ull;
+    }
+    const unsigned long long a = a0 + a1;
+    // warp sum of 64-bit values as three integer reductions of 22-bit limbs (one instruction each)
+    const unsigned r0 = __reduce_add_sync(0xffffffffu, (unsigned)(a & 0x3fffffull));
+    const unsigned r1 = __reduce_add_sync(0xffffffffu, (unsigned)((a >> 22) & 0x3fffffull));
+    const unsigned r2 = __reduce_add_sync(0xffffffffu, (unsigned)(a >> 44));
+    return (unsigned long long)r0 + ((unsigned long long)r1 << 22) + ((unsigned long long)r2 << 44);
+  };
+
+  const unsigned long long target =
+      (fixed_count > 0) ? (unsigned long long)min(fixed_count, nKb)
+                        : (unsigned long long)(fmin(tau, 1.0) * 1152921504606846976.0);
+  int s = nKb, need = 0;
+  uint32_t v = 0u;  // kept: bits > v, and the first `need` (by index) with bits == v
+  const bool all = (fixed_count <= 0 && tau >= 1.0) || measure_ge(0u) < target;  // never reaches tau
+  if (!all) {
+    for (int b = 30; b >= 0; --b) {
+      const uint32_t cand = v | (1u << b);
+      if (measure_ge(cand) >= target) v = cand;
+    }
+    unsigned long long gt = 0ull;
+    int n_gt = 0, n_eq = 0;
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+      const bool valid = (k * 32 + lane) < nKb;
+      if (valid && bits[k] > v) {
+        gt += fx[k];
+        ++n_gt;
+      }
+      if (valid && bits[k] == v) ++n_eq;
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      gt += __shfl_xor_sync(0xffffffffu, gt, d);
+      n_gt += __shfl_xor_sync(0xffffffffu, n_gt, d);
+      n_eq += __shfl_xor_sync(0xffffffffu, n_eq, d);
+    }
+    unsigned long long need64;
+    if (fixed_count > 0) {
+      need64 = target - gt;
+    } else {
+      const unsigned long long fv = (unsigned long long)((double)__uint_as_float(v) * 1152921504606846976.0);
+      need64 = (fv == 0ull) ? (unsigned long long)n_eq : (target - gt + fv - 1ull) / fv;
+    }
+    need = (int)min(need64, (unsigned long long)n_eq);
+    s = n_gt + need;
+  }
+  int seen = 0;  // ties at lower indices
+#pragma unroll
+  for (int k = 0; k < K; ++k) {
+    const bool valid = (k * 32 + lane) < nKb;
+    const bool eq = valid && !all && bits[k] == v;
+    const uint32_t eqm = __ballot_sync(0xffffffffu, eq);
+    const int rank = seen + __popc(eqm & ((1u << lane) - 1u));
+    const bool keep = valid && (all || bits[k] > v || (eq && rank < need));
+    seen += __popc(eqm);
+    const uint32_t word = __ballot_sync(0xffffffffu, keep);
+    if (lane == 0 && k < words) bitmaps[row * words + k] = word;
+  }
+  if (lane == 0) counts[row] = s;
 }
 
 __global__ void __launch_bounds__(1024)
@@ -250,15 +359,26 @@ int launch_select(int rows, int nKb, const float* mass, double tau, int fixed_co
   int32_t* counts = static_cast<int32_t*>(ws);
   uint32_t* bitmaps = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) +
                                                   align_up((size_t)rows * sizeof(int32_t), 256));
-  const int n2 = next_pow2(nKb);
-  const int words = (nKb + 31) / 32;
-  const size_t smem = (size_t)n2 * 8 + (size_t)words * 4;
-  if (smem > 48 * 1024) {
-    LOSA_CUDA_TRY(cudaFuncSetAttribute(select_rows_kernel,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  if (nKb <= 1024) {
+    // one warp per row, the row in registers, no sort
+    const int ctas = (rows + 3) / 4;
+    if (nKb <= 256)
+      select_rows_warp_kernel<8><<<ctas, 128, 0, st>>>(mass, rows, nKb, tau, fixed_count, counts, bitmaps, status);
+    else if (nKb <= 512)
+      select_rows_warp_kernel<16><<<ctas, 128, 0, st>>>(mass, rows, nKb, tau, fixed_count, counts, bitmaps, status);
+    else
+      select_rows_warp_kernel<32><<<ctas, 128, 0, st>>>(mass, rows, nKb, tau, fixed_count, counts, bitmaps, status);
+  } else {
+    const int n2 = next_pow2(nKb);
+    const int words = (nKb + 31) / 32;
+    const size_t smem = (size_t)n2 * 8 + (size_t)words * 4;
+    if (smem > 48 * 1024) {
+      LOSA_CUDA_TRY(cudaFuncSetAttribute(select_rows_kernel,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    }
+    select_rows_kernel<<<rows, kSelThreads, smem, st>>>(mass, nKb, n2, tau, fixed_count, counts, bitmaps,
+                                                        status);
   }
-  select_rows_kernel<<<rows, kSelThreads, smem, st>>>(mass, nKb, n2, tau, fixed_count, counts, bitmaps,
-                                                      status);
   scan_counts_kernel<<<1, 1024, 0, st>>>(counts, rows, offsets, kv_capacity, status);
   const int warps_per_cta = 8;
   expand_rows_kernel<<<(rows + warps_per_cta - 1) / warps_per_cta, warps_per_cta * 32, 0, st>>>(
