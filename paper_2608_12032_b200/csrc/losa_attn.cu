@@ -1244,7 +1244,7 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
   prm.nUnits = prm.nWork;
   prm.split_first = prm.nWork;
   prm.split_parts = 1;
-  if ((MODE == kDense || MODE == kSparse) && prm.nWork <= (int)kTlItemMask) {
+  if (MODE == kDense || MODE == kSparse) {
     const int rest = (prm.nWork < ctas) ? prm.nWork : prm.nWork % ctas;
     int parts = rest > 0 ? ctas / rest : 1;
     parts = min(min(parts, kMaxParts), prm.nKb);
@@ -1332,6 +1332,7 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
   prm.nQt = g.nQt;
   prm.nPairs = g.nPairs;
   prm.nWork = g.B * g.H * g.nPairs;
+  if (prm.nWork > (int)kTlItemMask) return LOSA_ERR_UNSUPPORTED;  // the tile list's item headers hold 24 bits
   prm.offsets = offsets;
   prm.kv_idx = kv_idx;
   prm.o = o;
