@@ -557,7 +557,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         flags = kTlPartial | ((uint32_t)part << 24);
       }
       const int unit = (flags != 0) ? p.split_first + (w - p.split_first) * parts + part : w;
-      const int bh = w / p.nPairs, pr = w % p.nPairs;
+      const int pr = w % p.nPairs;
       LOSA_TL_PUT(kTlItem | flags | (uint32_t)w);
       if (MODE == kSparse) {
         // the unit's merged tile list was built before the launch: stream it into the ring,
@@ -1011,7 +1011,6 @@ __global__ void __launch_bounds__(32) build_tile_lists_kernel(const Params p) {
   // left of the longer class.  Within a class the blocks ascend.  Correctness does not depend on
   // the order of the key blocks.
   uint32_t* dst = p.tl_entries + (int64_t)unit * p.tl_cap;
-  constexpr uint32_t kMaskA = (1u << (NB / 2)) - 1u;
   int nb = 0, na = 0, nbb = 0;  // both, tile 0 only, tile 1 only
   for (int w0 = 0; w0 < W; w0 += 32) {
     const int wi = w0 + lane;
