@@ -406,13 +406,22 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const uint32_t v_lo = ptx::smem_desc_lo(ptx::smem_u32(sV), C::kKVSlab);
       const uint32_t tS = tmem_base + qt * kSStride;
       const uint32_t tO = tmem_base + 256 + qt * 128;
-      // every descriptor is built before the waits, so that the MMAs issue back to back
-      uint64_t qd[D / 16];
+      // Every descriptor is built before the waits, so that the MMAs issue back to back.  The
+      // dense and sparse forward keep only the low words in registers (the high word is the same
+      // constant for every operand): 24 whole descriptors do not fit this warp's 72 registers
+      // and spilled, which cost 4 % of the forward.  The mass pass has half as many operands,
+      // and it and the fused mode were measured 3 % faster with whole descriptors.
+      constexpr bool kLoDesc = C::kHasV && !C::kWantMass;
+      uint32_t qd[D / 16];
 #pragma unroll
       for (int kk = 0; kk < D / 16; ++kk)
-        qd[kk] = ptx::desc64(ptx::smem_desc_lo(ptx::smem_u32(sQ), 16) + qt * (C::kQBytes >> 4) +
-                                 (((kk >> 2) * C::kQSlab + (kk & 3) * 32) >> 4),
-                             kDescHi);
+        qd[kk] = ptx::smem_desc_lo(ptx::smem_u32(sQ), 16) + qt * (C::kQBytes >> 4) +
+                 (((kk >> 2) * C::kQSlab + (kk & 3) * 32) >> 4);
+      uint64_t qd64[D / 16];
+      if (!kLoDesc) {
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) qd64[kk] = ptx::desc64(qd[kk], kDescHi);
+      }
 
       LOSA_TL_NEXT(ent);
       while ((ent >> 28) == 1) {
@@ -436,15 +445,22 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const uint32_t vs = nt % kNVs, vph = (nt / kNVs) & 1;
           const bool member = more && ((memb >> (qt * kQBT)) & kQMask) != 0;
           const uint32_t buf = nsub % kNS;
-          uint64_t kd[D / 16], vd[kW / 16];
+          uint32_t kd[D / 16], vd[kW / 16];
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk)
-            kd[kk] = ptx::desc64(k_lo + ks * (C::kKVBytes >> 4) +
-                                     (((kk >> 2) * C::kKVSlab + (kk & 3) * 32) >> 4),
-                                 kDescHi);
+            kd[kk] = k_lo + ks * (C::kKVBytes >> 4) + (((kk >> 2) * C::kKVSlab + (kk & 3) * 32) >> 4);
 #pragma unroll
           for (int kk = 0; kk < kW / 16; ++kk)
-            vd[kk] = ptx::desc64(v_lo + pend_vs * (C::kKVBytes >> 4) + kk * (2048 >> 4), kDescHi);
+            vd[kk] = v_lo + pend_vs * (C::kKVBytes >> 4) + kk * (2048 >> 4);
+          uint64_t kd64[D / 16], vd64[kW / 16];
+          if (!kLoDesc) {
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) kd64[kk] = ptx::desc64(kd[kk], kDescHi);
+            if (C::kHasV) {
+#pragma unroll
+              for (int kk = 0; kk < kW / 16; ++kk) vd64[kk] = ptx::desc64(vd[kk], kDescHi);
+            }
+          }
           // operands first, the softmax hand-over last: it is the wait that ends latest
           if (more) LOSA_WAIT(&ctl->k_full[ks], kph);
           if (member) {
@@ -478,16 +494,30 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             if (leader) {
               if (C::kHasV && pend) {
                 // O += P V for the previous key tile of this query tile
-                ptx::mma_ts_d(tO, tS, vd[0], C::kIdescPV, pv_item > 0 ? 1u : 0u);
+                if (kLoDesc) {
+                  ptx::mma_ts_lo(tO, tS, vd[0], kDescHi, C::kIdescPV, pv_item > 0 ? 1u : 0u);
 #pragma unroll
-                for (int kk = 1; kk < kW / 16; ++kk)
-                  ptx::mma_ts_d(tO, tS + kk * 8, vd[kk], C::kIdescPV, 1u);
+                  for (int kk = 1; kk < kW / 16; ++kk)
+                    ptx::mma_ts_lo(tO, tS + kk * 8, vd[kk], kDescHi, C::kIdescPV, 1u);
+                } else {
+                  ptx::mma_ts_d(tO, tS, vd64[0], C::kIdescPV, pv_item > 0 ? 1u : 0u);
+#pragma unroll
+                  for (int kk = 1; kk < kW / 16; ++kk)
+                    ptx::mma_ts_d(tO, tS + kk * 8, vd64[kk], C::kIdescPV, 1u);
+                }
               }
               if (member) {
-                ptx::mma_ss_d(tS + buf * 128, qd[0], kd[0], C::kIdescQK, 0u);
+                if (kLoDesc) {
+                  ptx::mma_ss_lo(tS + buf * 128, qd[0], kd[0], kDescHi, C::kIdescQK, 0u);
 #pragma unroll
-                for (int kk = 1; kk < D / 16; ++kk)
-                  ptx::mma_ss_d(tS + buf * 128, qd[kk], kd[kk], C::kIdescQK, 1u);
+                  for (int kk = 1; kk < D / 16; ++kk)
+                    ptx::mma_ss_lo(tS + buf * 128, qd[kk], kd[kk], kDescHi, C::kIdescQK, 1u);
+                } else {
+                  ptx::mma_ss_d(tS + buf * 128, qd64[0], kd64[0], C::kIdescQK, 0u);
+#pragma unroll
+                  for (int kk = 1; kk < D / 16; ++kk)
+                    ptx::mma_ss_d(tS + buf * 128, qd64[kk], kd64[kk], C::kIdescQK, 1u);
+                }
                 // completes after every MMA issued so far, the tile's last O += P V included
                 ptx::mma_commit(&ctl->s_full[qt][buf]);
               }
@@ -654,10 +684,15 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         TR(2, nsub);
         ptx::tc_fence_after_sync();
         uint32_t sr[kW];
+        // On the common path (a reference exists, no key of the tile is missing) only the first
+        // 32 columns are waited for here; the rest arrive while those are exponentiated.
+        const bool stream = C::kHasV && mine && have_ref && !ragged;
         if (mine) {
+          ptx::tmem_ld32(tSb, &sr[0]);
+          if (stream) ptx::tmem_wait_ld();
 #pragma unroll
-          for (int c0 = 0; c0 < kW; c0 += 32) ptx::tmem_ld32(tSb + c0, &sr[c0]);
-          ptx::tmem_wait_ld();
+          for (int c0 = 32; c0 < kW; c0 += 32) ptx::tmem_ld32(tSb + c0, &sr[c0]);
+          if (!stream) ptx::tmem_wait_ld();
         }
         TR(3, nsub);
         if (!C::kHasV) {
@@ -749,6 +784,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
 #pragma unroll
             for (int c = 0; c < kW; c += 4) {
+              if (C::kHasV && c == 32) ptx::tmem_wait_ld();  // (nothing is in flight on a second pass)
               float2 x0 = ptx::fma2(
                   make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2[c / kC]);
               float2 x1 = ptx::fma2(
