@@ -41,7 +41,7 @@ UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one sparse-forward launch, from the ncu capture
 # summarised in profiles/losa_attn_kernel_wan_ncu.md (not re-measured by this script)
-NCU_DRAM_BYTES_PER_LAUNCH = {"wan": 0.304345e9 + 0.088818e9}
+NCU_DRAM_BYTES_PER_LAUNCH = {"wan": 0.305036e9 + 0.086246e9}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
