@@ -163,6 +163,47 @@ def test_chain_mass_select_sparse_on_named_workloads(name, taus):
     assert losa.losa_async_status() == 0
 
 
+def test_two_guidance_branches_in_one_batch_keep_their_own_patterns():
+    """The two classifier-free-guidance branches travel as B = 2 and each (b, h, query block) row
+    of the CSR is its own pattern: one batched pass over both branches must equal the two
+    single-branch passes bit for bit (masses, CSR, output), and each branch must match the oracle
+    on its own pattern.  The branches get differently sharp scores, so their patterns differ."""
+    losa = lib()
+    H, N, D, BLK, tau = 2, 900, 128, 128, 0.9
+    q0, k0, v0 = make(1, H, N, D, 71, 1.0)
+    q1, k1, v1 = make(1, H, N, D, 81, 2.0)
+    q, k, v = (torch.cat(p) for p in ((q0, q1), (k0, k1), (v0, v1)))
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    mass = losa.losa_block_mass(qd, kd, BLK, BLK)
+    off, idx = losa.losa_select(mass, tau)
+    o = losa.losa_sparse_attn(qd, kd, vd, off, idx, BLK, BLK, out_dtype=torch.float32)
+    assert losa.losa_async_status() == 0
+    off_h, idx_h = off.cpu().numpy(), idx.cpu().numpy()
+    nQb = -(-N // BLK)
+    rows = H * nQb
+    per_branch = []
+    for b in range(2):
+        qb, kb, vb = (t[b:b + 1].contiguous() for t in (qd, kd, vd))
+        mb = losa.losa_block_mass(qb, kb, BLK, BLK)
+        ob_, ib_ = losa.losa_select(mb, tau)
+        o_b = losa.losa_sparse_attn(qb, kb, vb, ob_, ib_, BLK, BLK, out_dtype=torch.float32)
+        assert torch.equal(mb.reshape(-1), mass[b].reshape(-1))
+        lo, hi = off_h[b * rows], off_h[(b + 1) * rows]
+        assert np.array_equal(ob_.cpu().numpy(), off_h[b * rows:(b + 1) * rows + 1] - lo)
+        assert np.array_equal(ib_.cpu().numpy()[: hi - lo], idx_h[lo:hi])
+        assert torch.equal(o_b[0], o[b])
+        per_branch.append(util.csr_rows(ob_.cpu().numpy(), ib_.cpu().numpy()[: hi - lo]))
+        # against the oracle, branch by branch
+        qn, kn, vn = (util.to_np(t[b:b + 1]) for t in (q, k, v))
+        sel = orc.select(mb.cpu().numpy().reshape(rows, -1).astype(np.float64), tau)
+        bad, _ = util.compare_csr(ob_.cpu().numpy(), ib_.cpu().numpy(), sel)
+        assert not bad
+        ref = orc.blocks_to_tokens(
+            orc.sparse_attn(qn, kn, vn, BLK, BLK, sel.offsets, sel.kv_idx), 1, H, N)
+        util.assert_output_close(o[b:b + 1], ref, f"branch {b}")
+    assert per_branch[0] != per_branch[1]
+
+
 def test_strided_heads_layout():
     """[B, N, H, D] storage viewed as [B, H, N, D]: strides come from the problem description."""
     losa = lib()
