@@ -57,6 +57,28 @@ def test_select_ties_uniform_and_zero_masses():
         assert status == 0 and not util.compare_csr(off, idx, sel)[0]
 
 
+@pytest.mark.parametrize("nKb", [3, 8, 64, 2048])
+def test_select_threshold_is_inclusive_on_exactly_representable_masses(nKb):
+    """A prefix whose mass equals tau exactly already suffices (Eq. 3: >= tau).  Masses are powers
+    of two, so both sides add them without rounding; nKb = 2048 takes the sorting kernel."""
+    m = np.zeros((3, nKb), dtype=np.float32)
+    m[0, :3] = (0.5, 0.25, 0.25)
+    m[1, :3] = (0.25, 0.25, 0.5)
+    m[2, -1], m[2, 0], m[2, 1] = 0.5, 0.25, 0.25
+    for tau, counts in ((0.75, (2, 2, 2)), (0.5, (1, 1, 1)), (float(np.nextafter(0.5, 1.0)), (2, 2, 2))):
+        off, idx, status = run_select(m, tau)
+        sel = orc.select(m.astype(np.float64), tau)
+        assert status == 0
+        assert tuple(sel.count) == counts
+        bad, exempt = util.compare_csr(off, idx, sel)
+        # exact ties with tau sit inside the near-threshold band by definition: compare them anyway
+        assert util.csr_rows(off, idx[: off[-1]]) == util.csr_rows(sel.offsets, sel.kv_idx), (tau, bad, exempt)
+    if nKb == 8:
+        u = np.full((2, 8), 0.125, dtype=np.float32)
+        off, idx, status = run_select(u, 0.75)
+        assert status == 0 and list(np.diff(off)) == [6, 6] and list(idx[:6]) == list(range(6))
+
+
 def test_select_is_deterministic_and_multi_head():
     m32 = random_mass(2 * 3 * 16, 70, 5)
     a = run_select(m32, 0.9, B=2, H=3)

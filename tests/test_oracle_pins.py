@@ -192,6 +192,29 @@ def test_select_ties_broken_by_lower_index():
     assert sel.count[0] == 4 and list(sel.kept[0, :4]) == [0, 1, 2, 4]
 
 
+def test_select_threshold_is_inclusive():
+    """Eq. 3 keeps the shortest prefix whose mass is >= tau: a prefix that lands exactly on tau
+    already suffices.  Masses and thresholds are exactly representable, so equality is exact."""
+    m = np.array([[0.5, 0.25, 0.25], [0.25, 0.25, 0.5], [0.125, 0.5, 0.375]])
+    sel = orc.select(m, 0.75)
+    # row 0: 0.5 + 0.25 == 0.75 -> two blocks, the tie goes to the lower index
+    assert sel.count[0] == 2 and list(sel.kept[0, :2]) == [0, 1]
+    # row 1: order (2, 0, 1) with the tie by index; 0.5 + 0.25 == 0.75 -> {0, 2}
+    assert list(sel.order[1]) == [2, 0, 1]
+    assert sel.count[1] == 2 and list(sel.kept[1, :2]) == [0, 2]
+    # row 2: 0.5 + 0.375 = 0.875 >= 0.75 -> {1, 2}
+    assert sel.count[2] == 2 and list(sel.kept[2, :2]) == [1, 2]
+    assert np.all(sel.cum[:2, 1] == 0.75)
+    # a single block that equals tau suffices; one ulp more does not
+    sel = orc.select(np.array([[0.5, 0.25, 0.25]]), 0.5)
+    assert sel.count[0] == 1 and sel.kept[0, 0] == 0
+    sel = orc.select(np.array([[0.5, 0.25, 0.25]]), np.nextafter(0.5, 1.0))
+    assert sel.count[0] == 2
+    # uniform masses on a multiple of 1/nKb: 8 * 0.125 == 1.0 exactly, 6 * 0.125 == 0.75
+    sel = orc.select(np.full((1, 8), 0.125), 0.75)
+    assert sel.count[0] == 6 and list(sel.kept[0, :6]) == list(range(6))
+
+
 def test_select_one_hot_and_tau_one():
     m = np.zeros((2, 7))
     m[0, 4] = 1.0
