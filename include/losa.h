@@ -18,8 +18,11 @@
  * --------------------------------
  *  - All tensor pointers are DEVICE pointers on the current CUDA device,
  *    16-byte aligned.  The caller owns every buffer, including workspace;
- *    the library allocates no device memory per call (it keeps one small
- *    pinned status word and cached device properties per process).
+ *    the library allocates no device memory per call (per device it keeps
+ *    one small pinned status word and the SM count, created on the device's
+ *    first call).  Several devices may be driven from one process, each
+ *    call with its device current; a device that is not an sm_100 GPU gets
+ *    LOSA_ERR_UNSUPPORTED.
  *  - q, k, v, o are [B, H, N, D] with element strides (sb, sh, sn) and D
  *    contiguous; strides must be multiples of 8 elements.  q, k, v are bf16.
  *    N is the number of VALID tokens and need not be a multiple of the block
@@ -31,11 +34,16 @@
  *    stream) and return without synchronising.  The return value reports
  *    errors found on the host before any launch.  Errors found on the device
  *    (a bounded wait that expired, a bad block index, a negative mass, a CSR
- *    that overflowed its capacity) are recorded in a status word that
- *    losa_async_status() returns and clears.  No kernel ever traps, asserts
- *    or waits without a bound.
+ *    that overflowed its capacity) are recorded in the device's status word,
+ *    which losa_async_status() returns and clears.  The word is shared by
+ *    every stream and host thread that uses the device: it holds the first
+ *    error since it was last cleared, whichever call raised it.  No kernel
+ *    ever traps, asserts or waits without a bound.
  *  - Supported shapes: D in {64, 128}; (R, C) in {(64, 64), (128, 128), (128, 64), (128, 32)}
- *    (the last is the block geometry the paper runs with); fewer than 65535 key blocks.
+ *    (the last is the block geometry the paper runs with); fewer than 65535 key blocks for the
+ *    attention and mass calls, at most LOSA_SELECT_MAX_KEY_BLOCKS (8192) per row for the
+ *    selection calls (a longer row gets LOSA_ERR_UNSUPPORTED): with C = 32 the whole chain
+ *    mass -> select -> sparse attention therefore reaches 262144 tokens.
  */
 #ifndef LOSA_H_
 #define LOSA_H_
@@ -56,7 +64,8 @@ enum {
   LOSA_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed                            */
   LOSA_ERR_TIMEOUT = -6,     /* a bounded device-side wait expired (device-side)             */
   LOSA_ERR_BAD_INDEX = -7,   /* kv_idx / offsets out of range or not ascending (device-side) */
-  LOSA_ERR_BAD_MASS = -8     /* negative, NaN or > 8 mass seen by losa_select (device-side)  */
+  LOSA_ERR_BAD_MASS = -8     /* losa_select saw a negative, NaN or > 8 mass, or a row whose
+                                masses add up to more than 8 (device-side)                   */
 };
 
 enum {
@@ -68,6 +77,9 @@ enum {
 };
 
 enum { LOSA_DTYPE_BF16 = 0, LOSA_DTYPE_F32 = 1 };
+
+/* Longest mass row (key blocks) the selection calls accept. */
+#define LOSA_SELECT_MAX_KEY_BLOCKS 8192
 
 typedef struct {
   int32_t B, H, N, D; /* batch, heads, VALID tokens, head dimension                     */
@@ -87,8 +99,10 @@ size_t losa_workspace_bytes(int op, const losa_problem_t* p);
  *     A = row-wise softmax(q k^T * scale) over the N valid keys,
  * i.e. the paper's M(i,j) divided by the number of valid rows of query block i, so
  * that each row of `mass` sums to 1 and Eq. 3's threshold theta*R becomes tau.
- * The softmax is computed with a running maximum and sum; the per-key-block sums are
- * taken in the same pass.
+ * One pass over Q K^T: every row keeps a running sum of exponentials against a reference
+ * score that is raised whenever a tile's sums leave the safe range (for C < 128 the running
+ * maximum itself); the per-key-block sums are taken in the same pass and normalised by the
+ * row's final sum at the end.
  *   q, k    bf16 [B,H,N,D] (strides from p)
  *   mass    f32  [B,H,nQb,nKb] contiguous, fully overwritten
  *   lse     f32  [B,H,N] contiguous or NULL: natural-log sum-exp of each row's scaled scores
@@ -100,7 +114,9 @@ int losa_block_mass(const losa_problem_t* p, const void* q, const void* k, float
  * decreasing order (equal masses: lower block index first), accumulate them in fp64 and
  * keep the shortest prefix whose sum is >= tau; tau >= 1 keeps every block, and so does a
  * row whose sum never reaches tau.  Each row keeps at least one block.
- *   mass        f32 [rows, nKb], rows = B*H*nQb, values >= 0
+ *   mass        f32 [rows, nKb], rows = B*H*nQb, nKb <= LOSA_SELECT_MAX_KEY_BLOCKS; values in
+ *               [0, 8] and row sums <= 8 (a mass row sums to 1), else LOSA_ERR_BAD_MASS is
+ *               recorded: a bad value counts as 0, a row with a bad sum keeps every block
  *   tau         in (0, 1]
  *   offsets     i32 [rows + 1]: exclusive prefix of the per-row counts; offsets[rows] = nnz
  *   kv_idx      i32 [kv_capacity]: kept block indices, row after row, ascending in a row
@@ -142,7 +158,7 @@ int losa_row_recall(int32_t rows, int32_t nKb, const float* mass, const int32_t*
  * no cudaMalloc, cudaFree, cudaHostAlloc or other allocating call, and unlike the other entry
  * points it does not touch the library's pinned status word (creating that allocates).
  *
- * Same computation, arguments and results as losa_select, except:
+ * Same kernels, arguments and results as losa_select, except:
  *   - no workspace arguments.  The problem must fit the array: 256-byte-rounded 4*rows
  *     plus 4*rows*ceil(nKb/32) bytes, plus 256, at most LOSA_SELECT_NOALLOC_MAX_SCRATCH
  *     (all five benchmark shapes fit); otherwise LOSA_ERR_WORKSPACE is returned, nothing is
@@ -177,6 +193,39 @@ int losa_sparse_attn(const losa_problem_t* p, const void* q, const void* k, cons
                      const int32_t* offsets, const int32_t* kv_idx, void* o, int o_dtype,
                      void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* One problem of a batched launch: its tensors, its own frozen pattern, its output.  All
+ * problems of a launch share the shape, strides and block geometry of one losa_problem_t. */
+typedef struct {
+  const void* q;          /* bf16 [B,H,N,D] */
+  const void* k;
+  const void* v;
+  const int32_t* offsets; /* i32 [B*H*nQb + 1]: this problem's CSR */
+  const int32_t* kv_idx;
+  void* o;                /* [B,H,N,D], bf16 or f32 */
+} losa_layer_t;
+
+#define LOSA_MAX_BATCHED_LAYERS 64
+
+/* losa_sparse_attn (Eq. 4) for several problems in ONE persistent launch.  The paper keeps the
+ * pattern separately for each layer, head and query block and for the two guidance branches
+ * ("One-Time Pattern Construction"); the batch dimension B carries branches inside a call, this
+ * call carries whole problems that each have their own tensors and CSR - layers whose inputs
+ * are all available, or independent requests of one shape.  The persistent CTAs draw work
+ * items across all problems from one counter, so that small problems share one launch (a
+ * call on a 2048-token layer is bound by launch latency, not by work) and only the last wave
+ * of the whole batch, not of every problem, runs partly filled.  Each problem's result is bit
+ * for bit that of its own losa_sparse_attn call as long as neither launch cuts the work
+ * items of its last wave into parts (which items are cut depends on the total count).
+ *   layers   HOST array of n_layers entries (1 .. LOSA_MAX_BATCHED_LAYERS), device pointers
+ *            inside, 16-byte aligned; read before the call returns
+ *   ws       >= losa_workspace_bytes_batched(LOSA_OP_SPARSE_ATTN, p, n_layers) bytes,
+ *            128-byte aligned */
+int losa_sparse_attn_batched(const losa_problem_t* p, int32_t n_layers, const losa_layer_t* layers,
+                             int o_dtype, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Workspace of a batched call (op: LOSA_OP_SPARSE_ATTN); 0 for an invalid problem or count. */
+size_t losa_workspace_bytes_batched(int op, const losa_problem_t* p, int32_t n_layers);
+
 /* Dense softmax attention o = softmax(q k^T * scale) v over the N valid keys: the paper's
  * dense steps up to the construction step, and this library's own dense baseline.
  * Same tensors and workspace rule as losa_sparse_attn, without the CSR. */
@@ -184,9 +233,8 @@ int losa_attn(const losa_problem_t* p, const void* q, const void* k, const void*
               int o_dtype, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* The construction step as one kernel: dense attention that also accumulates the exact block
- * masses (the paper's implementation builds the pattern with "a custom dense-attention kernel
- * that accumulates exact block masses while computing full attention", Implementation
- * paragraph; pattern construction coincides with the dense step t0).  Results are those of
+ * masses (the paper's Implementation paragraph builds the pattern inside the dense attention of
+ * step t0, with a kernel of its own that sums the block masses on the way).  Results are those of
  * losa_attn (o) and losa_block_mass (mass, optional lse) on the same inputs, from one pass over
  * Q K^T.
  *   ws   >= losa_workspace_bytes(LOSA_OP_ATTN_MASS, p) bytes                               */
@@ -204,6 +252,17 @@ int losa_validate_csr(int32_t rows, int32_t nKb, const int32_t* offsets, const i
 /* Synchronises `cuda_stream`, then returns and clears the device-side status word
  * (LOSA_OK or the first device-side LOSA_ERR_* recorded since the last call). */
 int losa_async_status(void* cuda_stream);
+
+/* Diagnostic for tests of the time-out path.  (The paper has no counterpart.)  Every wait inside
+ * the attention kernels is bounded; this call makes the bound observable without harming the
+ * GPU.  It arms ONE launch: the next losa_attn, losa_sparse_attn, losa_block_mass or
+ * losa_attn_mass of this process runs its kernel with the role that publishes the work
+ * (the tile lists) publishing nothing, and with every device-side wait limited to `polls` polls
+ * (1 .. 65536; a few milliseconds) instead of about a second.  No copy and no tensor-core
+ * instruction is issued in that launch; every role's first wait runs out, the CTAs leave through
+ * the common teardown that frees tensor memory, and the status word becomes LOSA_ERR_TIMEOUT.
+ * The outputs of that call are undefined.  The launch after it is an ordinary one. */
+int losa_debug_stall_next_launch(uint32_t polls);
 
 /* Static, human-readable name of a status code. */
 const char* losa_status_string(int status);

@@ -10,13 +10,16 @@ from .binding import (  # noqa: F401
     losa_attn,
     losa_attn_mass,
     losa_block_mass,
+    losa_debug_stall_next_launch,
     losa_select,
     losa_select_noalloc,
     losa_select_topk,
     losa_row_recall,
     losa_sparse_attn,
+    losa_sparse_attn_batched,
     losa_status_string,
     losa_validate_csr,
     losa_workspace_bytes,
+    losa_workspace_bytes_batched,
     make_problem,
 )

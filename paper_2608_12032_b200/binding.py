@@ -23,6 +23,7 @@ EXPORTS = (
     "losa_workspace_bytes", "losa_block_mass", "losa_select", "losa_sparse_attn", "losa_attn",
     "losa_attn_mass", "losa_select_topk", "losa_row_recall",
     "losa_select_noalloc", "losa_validate_csr", "losa_async_status", "losa_status_string", "losa_last_cuda_error",
+    "losa_debug_stall_next_launch", "losa_sparse_attn_batched", "losa_workspace_bytes_batched",
 )
 
 
@@ -41,6 +42,13 @@ class Problem(ctypes.Structure):
         ("R", ctypes.c_int32), ("C", ctypes.c_int32),
         ("sb", ctypes.c_int64), ("sh", ctypes.c_int64), ("sn", ctypes.c_int64),
         ("scale", ctypes.c_float),
+    ]
+
+
+class Layer(ctypes.Structure):
+    _fields_ = [
+        ("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p),
+        ("offsets", ctypes.c_void_p), ("kv_idx", ctypes.c_void_p), ("o", ctypes.c_void_p),
     ]
 
 
@@ -72,6 +80,10 @@ def _lib():
         lib.losa_select_noalloc.argtypes = [i32, i32, i32, i32, vp, ctypes.c_double, vp, vp, i64, vp, vp]
         lib.losa_sparse_attn.restype = ctypes.c_int
         lib.losa_sparse_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, ctypes.c_int, vp, sz, vp]
+        lib.losa_sparse_attn_batched.restype = ctypes.c_int
+        lib.losa_sparse_attn_batched.argtypes = [pp, i32, ctypes.POINTER(Layer), ctypes.c_int, vp, sz, vp]
+        lib.losa_workspace_bytes_batched.restype = sz
+        lib.losa_workspace_bytes_batched.argtypes = [ctypes.c_int, pp, i32]
         lib.losa_attn.restype = ctypes.c_int
         lib.losa_attn.argtypes = [pp, vp, vp, vp, vp, ctypes.c_int, vp, sz, vp]
         lib.losa_attn_mass.restype = ctypes.c_int
@@ -80,6 +92,8 @@ def _lib():
         lib.losa_validate_csr.argtypes = [i32, i32, vp, vp, vp]
         lib.losa_async_status.restype = ctypes.c_int
         lib.losa_async_status.argtypes = [vp]
+        lib.losa_debug_stall_next_launch.restype = ctypes.c_int
+        lib.losa_debug_stall_next_launch.argtypes = [ctypes.c_uint32]
         lib.losa_status_string.restype = ctypes.c_char_p
         lib.losa_status_string.argtypes = [ctypes.c_int]
         lib.losa_last_cuda_error.restype = ctypes.c_char_p
@@ -236,6 +250,34 @@ def losa_sparse_attn(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, offsets:
     return o
 
 
+def losa_workspace_bytes_batched(op: int, problem: Problem, n_layers: int) -> int:
+    return int(_lib().losa_workspace_bytes_batched(op, ctypes.byref(problem), int(n_layers)))
+
+
+def losa_sparse_attn_batched(layers, R: int, C: int, scale: Optional[float] = None,
+                             out_dtype: torch.dtype = torch.bfloat16, outs=None,
+                             ws: Optional[torch.Tensor] = None):
+    """Block-sparse attention of several problems of one shape in one launch.
+
+    ``layers`` is a sequence of ``(q, k, v, offsets, kv_idx)``; returns the list of outputs."""
+    q0 = layers[0][0]
+    prob = make_problem(q0, R, C, scale)
+    arr = (Layer * len(layers))()
+    result = []
+    for i, (q, k, v, offsets, kv_idx) in enumerate(layers):
+        _same_layout(q0, q, k, v)
+        o = _alloc_out(q, out_dtype, None if outs is None else outs[i])
+        result.append(o)
+        arr[i] = Layer(_ptr(q), _ptr(k), _ptr(v), _ptr(offsets), _ptr(kv_idx), _ptr(o))
+    need = losa_workspace_bytes_batched(LOSA_OP_SPARSE_ATTN, prob, len(layers))
+    if ws is None:
+        ws = torch.empty(max(need, 1), dtype=torch.uint8, device=q0.device)
+    _check(_lib().losa_sparse_attn_batched(ctypes.byref(prob), len(layers), arr,
+                                           _dtype_code(result[0].dtype), _ptr(ws), ws.numel(), _stream()),
+           "losa_sparse_attn_batched")
+    return result
+
+
 def losa_attn(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, R: int = 128, C: int = 128,
               scale: Optional[float] = None, out_dtype: torch.dtype = torch.bfloat16,
               out: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None):
@@ -276,6 +318,11 @@ def losa_validate_csr(offsets: torch.Tensor, kv_idx: torch.Tensor, nKb: int) -> 
 def losa_async_status() -> int:
     """Synchronises the current stream and returns (and clears) the device-side status."""
     return int(_lib().losa_async_status(_stream()))
+
+
+def losa_debug_stall_next_launch(polls: int = 2048) -> None:
+    """Arms one diagnostic attention launch whose waits all run out (LOSA_ERR_TIMEOUT)."""
+    _check(_lib().losa_debug_stall_next_launch(int(polls)), "losa_debug_stall_next_launch")
 
 
 def losa_status_string(code: int) -> str:

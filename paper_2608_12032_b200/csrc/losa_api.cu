@@ -3,14 +3,19 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "losa_common.cuh"
 
 namespace losa {
 
 namespace {
 thread_local char g_cuda_error[256] = "";
-int* g_status_host = nullptr;
-int* g_status_dev = nullptr;
+std::mutex g_state_mutex;
+DeviceState g_state[kMaxDevices];
+std::atomic<int> g_state_ready[kMaxDevices];  // 0 = not created, 1 = ready
+std::atomic<int> g_device_ok[kMaxDevices];    // 0 = not asked, 1 = sm_100, -1 = anything else
 }  // namespace
 
 const char* set_cuda_error(cudaError_t e, const char* what) {
@@ -18,32 +23,57 @@ const char* set_cuda_error(cudaError_t e, const char* what) {
   return g_cuda_error;
 }
 
-// One pinned, mapped int per process; every CUDA device of a unified-addressing system can
-// reach it, so it is not per-device state.
-int* status_word_device() {
-  if (!g_status_dev) {
-    int* h = nullptr;
-    cudaError_t e = cudaHostAlloc(reinterpret_cast<void**>(&h), 64,
-                                  cudaHostAllocMapped | cudaHostAllocPortable);
-    if (e != cudaSuccess) {
-      set_cuda_error(e, "cudaHostAlloc(status word)");
-      return nullptr;
-    }
-    *h = 0;
-    int* d = nullptr;
-    e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&d), h, 0);
-    if (e != cudaSuccess) {
-      set_cuda_error(e, "cudaHostGetDevicePointer(status word)");
-      cudaFreeHost(h);
-      return nullptr;
-    }
-    g_status_host = h;
-    g_status_dev = d;
+int check_device() {
+  int dev = 0;
+  LOSA_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return LOSA_ERR_UNSUPPORTED;
+  int ok = g_device_ok[dev].load(std::memory_order_acquire);
+  if (ok == 0) {
+    int major = 0;
+    LOSA_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    ok = (major == 10) ? 1 : -1;  // the kernels are built for sm_100a only
+    g_device_ok[dev].store(ok, std::memory_order_release);
   }
-  return g_status_dev;
+  if (ok < 0) {
+    snprintf(g_cuda_error, sizeof(g_cuda_error),
+             "device %d is not an sm_100 GPU: liblosa holds sm_100a kernels only", dev);
+    return LOSA_ERR_UNSUPPORTED;
+  }
+  return LOSA_OK;
 }
 
-int* status_word_host() { return g_status_host; }
+const DeviceState* device_state(int* rc) {
+  int dev = 0;
+  *rc = check_device();
+  if (*rc != LOSA_OK) return nullptr;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    *rc = LOSA_ERR_CUDA;
+    return nullptr;
+  }
+  if (g_state_ready[dev].load(std::memory_order_acquire)) return &g_state[dev];
+  std::lock_guard<std::mutex> lock(g_state_mutex);
+  if (g_state_ready[dev].load(std::memory_order_acquire)) return &g_state[dev];
+  DeviceState st{};
+  cudaError_t e = cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess) {
+    int* h = nullptr;
+    e = cudaHostAlloc(reinterpret_cast<void**>(&h), 64, cudaHostAllocMapped | cudaHostAllocPortable);
+    if (e == cudaSuccess) {
+      *h = 0;
+      e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&st.status_dev), h, 0);
+      if (e != cudaSuccess) cudaFreeHost(h);
+      st.status_host = h;
+    }
+  }
+  if (e != cudaSuccess || st.sm_count <= 0) {
+    set_cuda_error(e, "per-device state (SM count, status word)");
+    *rc = LOSA_ERR_CUDA;
+    return nullptr;
+  }
+  g_state[dev] = st;
+  g_state_ready[dev].store(1, std::memory_order_release);
+  return &g_state[dev];
+}
 
 int make_geometry(const losa_problem_t* p, Geometry* g) {
   if (!p) return LOSA_ERR_INVALID_ARG;
@@ -122,12 +152,15 @@ int losa_select(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const float* mas
   if (!mass || !offsets || !kv_idx || kv_capacity < 0) return LOSA_ERR_INVALID_ARG;
   const int64_t rows = (int64_t)B * H * nQb;
   if (rows * nKb > INT32_MAX) return LOSA_ERR_UNSUPPORTED;
-  if (nKb > 8192) return LOSA_ERR_UNSUPPORTED;  // one row is sorted in shared memory
+  if (nKb > LOSA_SELECT_MAX_KEY_BLOCKS) return LOSA_ERR_UNSUPPORTED;  // one row is sorted in shared memory
   const size_t need = select_workspace_bytes(rows, nKb);
   if (!ws || ws_bytes < need) return LOSA_ERR_WORKSPACE;
   if (!aligned16(ws)) return LOSA_ERR_INVALID_ARG;
+  int rc = LOSA_OK;
+  const DeviceState* dev = device_state(&rc);
+  if (!dev) return rc;
   return launch_select((int)rows, nKb, mass, tau, 0, offsets, kv_idx, kv_capacity, ws,
-                       static_cast<cudaStream_t>(cuda_stream));
+                       dev->status_dev, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int losa_select_topk(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const float* mass, int32_t k,
@@ -137,12 +170,15 @@ int losa_select_topk(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const float
   if (k < 1 || k > nKb) return LOSA_ERR_INVALID_ARG;
   if (!mass || !offsets || !kv_idx || kv_capacity < 0) return LOSA_ERR_INVALID_ARG;
   const int64_t rows = (int64_t)B * H * nQb;
-  if (rows * nKb > INT32_MAX || nKb > 8192) return LOSA_ERR_UNSUPPORTED;
+  if (rows * nKb > INT32_MAX || nKb > LOSA_SELECT_MAX_KEY_BLOCKS) return LOSA_ERR_UNSUPPORTED;
   const size_t need = select_workspace_bytes(rows, nKb);
   if (!ws || ws_bytes < need) return LOSA_ERR_WORKSPACE;
   if (!aligned16(ws)) return LOSA_ERR_INVALID_ARG;
+  int rc = LOSA_OK;
+  const DeviceState* dev = device_state(&rc);
+  if (!dev) return rc;
   return launch_select((int)rows, nKb, mass, 0.5, k, offsets, kv_idx, kv_capacity, ws,
-                       static_cast<cudaStream_t>(cuda_stream));
+                       dev->status_dev, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int losa_row_recall(int32_t rows, int32_t nKb, const float* mass, const int32_t* offsets,
@@ -160,7 +196,7 @@ int losa_select_noalloc(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const fl
   if (!(tau > 0.0) || !(tau <= 1.0)) return LOSA_ERR_INVALID_ARG;
   if (!mass || !offsets || !kv_idx || kv_capacity < 0) return LOSA_ERR_INVALID_ARG;
   const int64_t rows = (int64_t)B * H * nQb;
-  if (rows * nKb > INT32_MAX || nKb > 8192) return LOSA_ERR_UNSUPPORTED;
+  if (rows * nKb > INT32_MAX || nKb > LOSA_SELECT_MAX_KEY_BLOCKS) return LOSA_ERR_UNSUPPORTED;
   const size_t need = select_workspace_bytes(rows, nKb);
   if (need > select_noalloc_workspace_limit()) {
     snprintf(g_cuda_error, sizeof(g_cuda_error),
@@ -169,6 +205,8 @@ int losa_select_noalloc(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const fl
              need, select_noalloc_workspace_limit());
     return LOSA_ERR_WORKSPACE;
   }
+  const int rc = check_device();  // (asks for an attribute; allocates nothing)
+  if (rc != LOSA_OK) return rc;
   return launch_select_noalloc((int)rows, nKb, mass, tau, offsets, kv_idx, kv_capacity,
                                device_status, static_cast<cudaStream_t>(cuda_stream));
 }
@@ -194,6 +232,33 @@ int losa_sparse_attn(const losa_problem_t* p, const void* q, const void* k, cons
   if (!aligned16(ws)) return LOSA_ERR_INVALID_ARG;
   return launch_attn(kSparse, g, q, k, v, offsets, kv_idx, o, o_dtype, nullptr, nullptr, ws,
                      static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t losa_workspace_bytes_batched(int op, const losa_problem_t* p, int32_t n_layers) {
+  Geometry g;
+  if (op != LOSA_OP_SPARSE_ATTN || n_layers < 1 || n_layers > LOSA_MAX_BATCHED_LAYERS) return 0;
+  if (make_geometry(p, &g) != LOSA_OK) return 0;
+  if ((int64_t)n_layers * g.B * g.H * g.nPairs > (int64_t)0x00ffffff) return 0;
+  return attn_workspace_bytes(kSparse, g, n_layers);
+}
+
+int losa_sparse_attn_batched(const losa_problem_t* p, int32_t n_layers, const losa_layer_t* layers,
+                             int o_dtype, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Geometry g;
+  if (n_layers < 1 || n_layers > LOSA_MAX_BATCHED_LAYERS || !layers) return LOSA_ERR_INVALID_ARG;
+  for (int i = 0; i < n_layers; ++i) {
+    const int rc = check_attn_args(p, &g, layers[i].q, layers[i].k, layers[i].v, layers[i].o, o_dtype);
+    if (rc != LOSA_OK) return rc;
+    if (!layers[i].offsets || !layers[i].kv_idx) return LOSA_ERR_INVALID_ARG;
+  }
+  if (!ws || ws_bytes < attn_workspace_bytes(kSparse, g, n_layers)) return LOSA_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(ws) & 127u) return LOSA_ERR_INVALID_ARG;
+  if (n_layers == 1)
+    return launch_attn(kSparse, g, layers[0].q, layers[0].k, layers[0].v, layers[0].offsets,
+                       layers[0].kv_idx, layers[0].o, o_dtype, nullptr, nullptr, ws,
+                       static_cast<cudaStream_t>(cuda_stream));
+  return launch_attn(kSparse, g, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, o_dtype, nullptr,
+                     nullptr, ws, static_cast<cudaStream_t>(cuda_stream), n_layers, layers);
 }
 
 int losa_attn(const losa_problem_t* p, const void* q, const void* k, const void* v, void* o,
@@ -232,11 +297,19 @@ int losa_async_status(void* cuda_stream) {
     set_cuda_error(e, "cudaStreamSynchronize");
     return LOSA_ERR_CUDA;
   }
-  int* h = status_word_host();
-  if (!h) return LOSA_OK;  // nothing was ever launched
-  const int s = *reinterpret_cast<volatile int*>(h);
-  *reinterpret_cast<volatile int*>(h) = 0;
-  return s;
+  // the word of the current device (the stream's device, by the calling convention); a device
+  // that never launched anything has none
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LOSA_ERR_CUDA;
+  if (!g_state_ready[dev].load(std::memory_order_acquire)) return LOSA_OK;
+  int* h = g_state[dev].status_host;
+  return __atomic_exchange_n(h, 0, __ATOMIC_ACQ_REL);
+}
+
+int losa_debug_stall_next_launch(uint32_t polls) {
+  if (polls == 0u || polls > (1u << 16)) return LOSA_ERR_INVALID_ARG;
+  arm_stalled_launch(polls);
+  return LOSA_OK;
 }
 
 const char* losa_status_string(int status) {

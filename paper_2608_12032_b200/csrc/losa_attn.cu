@@ -32,11 +32,16 @@
 #include <cuda_bf16.h>
 #include <math.h>
 
+#include <atomic>
+#include <vector>
+
 #include "losa_common.cuh"
 #include "losa_ptx.cuh"
 
 namespace losa {
 namespace {
+
+std::atomic<uint32_t> g_stall_polls{0u};  // > 0: the next attention launch is a diagnostic one
 
 constexpr int kThreads = 384;  // 2 softmax warpgroups + 1 utility warpgroup (TMA, 2 MMA issuers, scheduler)
 constexpr int kRegsSoftmax = 216, kRegsUtility = 72, kRegsAtLaunch = 168;
@@ -101,8 +106,23 @@ struct Cfg {
   static constexpr uint32_t kIdescPV = ptx::idesc_bf16_f32(128, D, false, true);
 };
 
+// One entry per problem of a batched launch (several layers or requests of one shape in one
+// persistent launch): the problem's tensor maps, its output and its own CSR pattern.  The table
+// lives in the workspace and is written by the host before the launch.
+struct alignas(128) ProblemEntry {
+  CUtensorMap map_q, map_k, map_v;
+  void* o;
+  const int32_t* offsets;
+  const int32_t* kv_idx;
+};
+
 struct Params {
   int B, H, N, nQb, nKb, nQt, nPairs, nWork;
+  // Batched launch: work items run over nProb problems, item w belongs to problem
+  // w / (B * H * nPairs); `problems` is null for a single problem, whose maps are kernel
+  // parameters and whose o / offsets / kv_idx are the fields below.
+  int nProb;
+  const ProblemEntry* problems;
   // Work units: items [0, split_first) whole, items [split_first, nWork) in split_parts parts of
   // their key-block lists each (the last, partly filled wave of the persistent grid is cut finer).
   int nUnits, split_first, split_parts;
@@ -125,6 +145,8 @@ struct Params {
   float2* table;  // mass modes: [grid][2][nKb][128] (sum of p, reference max) per row and key tile
   float scale_log2;
   int* status;
+  uint32_t wait_polls;  // bound of every device-side wait, in polls (ptx::kWaitPolls)
+  int stall;            // diagnostic launch: the scheduler publishes nothing, so that every wait runs out
 };
 
 template <int NK, int NV>
@@ -144,23 +166,9 @@ struct Control {
   int abort_flag;
 };
 
-// Event trace (diagnostic builds only, -DLOSA_TRACE): CTA 0 records (clock, event, counter) per role.
-#ifdef LOSA_TRACE
-__device__ unsigned long long g_trace[8][4096];
-#define TR_DECL(role) unsigned long long* tr_ = g_trace[role]; int tr_n = 0; const bool tr_on = (blockIdx.x == 0 && lane == 0)
-#define TR(ev, n)                                                                           \
-  do {                                                                                      \
-    if (tr_on && tr_n < 4096)                                                               \
-      tr_[tr_n++] = ((unsigned long long)clock64() << 24) | ((unsigned long long)((n) & 0xffff) << 8) | (ev); \
-  } while (0)
-#else
-#define TR_DECL(role) do {} while (0)
-#define TR(ev, n) do {} while (0)
-#endif
-
 #define LOSA_WAIT_RELAXED(bar, parity)                                   \
   do {                                                                   \
-    if (!ptx::mbar_wait_relaxed((bar), (parity), &ctl->abort_flag)) {    \
+    if (!ptx::mbar_wait_relaxed((bar), (parity), &ctl->abort_flag, p.wait_polls)) {    \
       ctl->abort_flag = 1;                                               \
       report_error(p.status, LOSA_ERR_TIMEOUT);                          \
       goto teardown;                                                     \
@@ -169,7 +177,7 @@ __device__ unsigned long long g_trace[8][4096];
 
 #define LOSA_WAIT(bar, parity)                                   \
   do {                                                           \
-    if (!ptx::mbar_wait((bar), (parity), &ctl->abort_flag)) {    \
+    if (!ptx::mbar_wait((bar), (parity), &ctl->abort_flag, p.wait_polls)) {    \
       ctl->abort_flag = 1;                                       \
       report_error(p.status, LOSA_ERR_TIMEOUT);                  \
       goto teardown;                                             \
@@ -318,8 +326,16 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       LOSA_TL_NEXT(ent);
       while ((ent >> 28) == 1) {
         const int w = (int)(ent & kTlItemMask);
-        const int bh = w / p.nPairs, pr = w % p.nPairs;
+        const int pbh = w / p.nPairs, pr = w % p.nPairs;
+        const int bh = pbh % (p.B * p.H);
         const int b = bh / p.H, h = bh % p.H;
+        const CUtensorMap *mq = &map_q, *mk = &map_k, *mv = &map_v;
+        if (p.problems != nullptr) {
+          const ProblemEntry* pe = p.problems + pbh / (p.B * p.H);
+          mq = &pe->map_q;
+          mk = &pe->map_k;
+          mv = &pe->map_v;
+        }
 #pragma unroll
         for (int qt = 0; qt < 2; ++qt) {
           const int T = 2 * pr + qt;
@@ -329,7 +345,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               ptx::mbar_arrive_expect_tx(&ctl->q_full[qt], C::kQBytes);
 #pragma unroll
               for (int s = 0; s < C::kDH; ++s)
-                ptx::tma_load_4d(sQ + qt * C::kQBytes + s * C::kQSlab, &map_q, &ctl->q_full[qt],
+                ptx::tma_load_4d(sQ + qt * C::kQBytes + s * C::kQSlab, mq, &ctl->q_full[qt],
                                  s * 64, T * 128, h, b);
             }
             ++nq[qt];
@@ -359,7 +375,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               if (g == gg) eg = grp[gg];
             const int jg = (int)(eg & 0xffffu);
             const int r0 = (jg == (int)kTlPad) ? p.nKb * kC : jg * kC;
-            ptx::tma_load_4d(sK + ks * C::kKVBytes + s * C::kKVSlab + g * C::kBoxBytes, &map_k,
+            ptx::tma_load_4d(sK + ks * C::kKVBytes + s * C::kKVSlab + g * C::kBoxBytes, mk,
                              &ctl->k_full[ks], s * 64, r0, h, b);
           }
           ++nk;
@@ -376,7 +392,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 if (g == gg) eg = grp[gg];
               const int jg = (int)(eg & 0xffffu);
               const int r0 = (jg == (int)kTlPad) ? p.nKb * kC : jg * kC;
-              ptx::tma_load_4d(sV + vs * C::kKVBytes + s * C::kKVSlab + g * C::kBoxBytes, &map_v,
+              ptx::tma_load_4d(sV + vs * C::kKVBytes + s * C::kKVSlab + g * C::kBoxBytes, mv,
                                &ctl->v_full[vs], s * 64, r0, h, b);
             }
             ++nv;
@@ -400,7 +416,6 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const int qt = warp - kIssuerWarp;
       const bool leader = (lane == 0);
       uint32_t nq = 0, nt = 0, nsub = 0, nof = 0, te = 0, ent;
-      TR_DECL(2 + qt);
       constexpr uint32_t kDescHi = ptx::smem_desc_hi_sw128(1024);
       const uint32_t k_lo = ptx::smem_desc_lo(ptx::smem_u32(sK), 16);
       const uint32_t v_lo = ptx::smem_desc_lo(ptx::smem_u32(sV), C::kKVSlab);
@@ -476,9 +491,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if (C::kHasV && pend) {
             LOSA_WAIT(&ctl->v_full[pend_vs], pend_vph);
             if (pv_item == 0 && nof > 0) LOSA_WAIT(&ctl->o_free[qt], (nof - 1) & 1);
-            TR(1, nsub);
             LOSA_WAIT(&ctl->p_ready[qt], (nsub - 1) & 1);
-            TR(2, nsub);
           }
           if ((C::kHasV && pend) || member) {
             // ---- one burst, under the lock
@@ -527,7 +540,6 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               if (C::kHasV && pend) ptx::mma_commit(&ctl->v_empty[pend_vs]);
               if (member) ptx::mma_commit(&ctl->k_empty[ks]);
             }
-            TR(3, nsub);
           }
           if (C::kHasV && pend) {
             ++pv_item;
@@ -570,6 +582,9 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // and the ascending merge of its tiles; nobody else touches the CSR.
     uint32_t te = 0;
     for (;;) {
+      // (diagnostic launch, see losa_debug_stall_next_launch: no tile list is ever published, no
+      // copy and no MMA is issued, and every other role's first wait runs out)
+      if (p.stall) break;
       // work items are drawn from a global counter, in head-major order, so that a CTA that
       // finishes early takes the next item instead of idling at the end of the launch
       int w = 0;
@@ -618,10 +633,12 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         LOSA_TL_PUT_BULK(e, n);
       }
     }
-    LOSA_TL_PUT(kTlEnd);
-    if ((te & 31) != 0) {  // publish the last, partly filled chunk
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&ctl->tl_full[((te - 1) >> 5) & (kTlChunks - 1)]);
+    if (!p.stall) {
+      LOSA_TL_PUT(kTlEnd);
+      if ((te & 31) != 0) {  // publish the last, partly filled chunk
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&ctl->tl_full[((te - 1) >> 5) & (kTlChunks - 1)]);
+      }
     }
   }
   } else {
@@ -636,18 +653,21 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int my_bit = qt * kQBT + sub;
     uint32_t nsub = 0, nwg = 0, nod = 0;      // nsub: key tiles of this query tile so far
     uint32_t te = 0, ent;
-    TR_DECL((wl == 0) ? qt : 7);
 
     LOSA_TL_NEXT(ent);
     while ((ent >> 28) == 1) {
       const int w = (int)(ent & kTlItemMask);
       const bool partial = (ent & kTlPartial) != 0;
       const int part = (int)((ent >> 24) & 7u);
-      const int bh = w / p.nPairs, pr = w % p.nPairs;
+      const int pbh = w / p.nPairs, pr = w % p.nPairs;
+      const int bh = pbh % (p.B * p.H);
       const int b = bh / p.H, h = bh % p.H;
+      void* const o_base = (p.problems != nullptr) ? p.problems[pbh / (p.B * p.H)].o : p.o;
       const int T = 2 * pr + qt;
       const int grow = T * 128 + row;
-      float m_ref = -INFINITY, l = 0.f;
+      // l: row sum of the exponentials; in the attention-only modes of their bf16 roundings (what
+      // the output is normalised by); the fused mode keeps both, the roundings' sum in lr
+      float m_ref = -INFINITY, l = 0.f, lr = 0.f;
       bool have_ref = false;  // this warp's rows have a reference maximum (after their first tile)
       uint32_t pv_item = 0;
       float2* tab = nullptr;
@@ -679,9 +699,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint32_t buf = nsub % kNS;
         const uint32_t tSb = tS + buf * 128;
         // S of this key tile is complete, and so is every earlier product into O
-        TR(1, nsub);
         LOSA_WAIT(&ctl->s_full[qt][buf], (nsub / kNS) & 1);
-        TR(2, nsub);
         ptx::tc_fence_after_sync();
         uint32_t sr[kW];
         // On the common path (a reference exists, no key of the tile is missing) only the first
@@ -694,7 +712,6 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           for (int c0 = 32; c0 < kW; c0 += 32) ptx::tmem_ld32(tSb + c0, &sr[c0]);
           if (!stream) ptx::tmem_wait_ld();
         }
-        TR(3, nsub);
         if (!C::kHasV) {
           // mass pass: S is in registers (and stays there: no P is packed over it), hand the
           // buffer back
@@ -712,7 +729,14 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           // O and the row sum, and exponentiate the tile again.  P is therefore stored only after
           // that test (S stays intact in TMEM for the second pass).
           float2 acc[kG][2];  // row sums per key block (the mass pass needs them apart), two chains each
-          float gsum[kG], tsum = 0.f;
+          // The output is normalised by the sum of the weights the tensor core actually multiplies
+          // with V - P as rounded to bf16 - not by the sum of the unrounded exponentials: then
+          // o = sum(p~ v) / sum(p~) is a weighted mean of V whatever the rounding does, exact for a
+          // row that one key dominates (with the unrounded sum such a row is off by up to 2^-8 |v|,
+          // because the reference is not the row maximum and the dominant p is not a power of two).
+          // The masses keep the unrounded sums.
+          float2 racc[2];
+          float gsum[kG], tsum = 0.f, rsum = 0.f;
           // (All rows of a warp belong to one query block and have seen the same tiles, so
           // whether a reference exists is known per warp without a vote.  In the mass pass the
           // scores stay in registers - no P is packed over them - so its second pass needs no
@@ -753,6 +777,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               const float alpha = need ? ptx::ex2_approx(m_ref - m_new) : 1.f;
               if (need) m_ref = m_new;
               l *= alpha;
+              lr *= alpha;
               if (C::kHasV && pv_item > 0) {
                 // (every earlier product into O is complete: s_full covers them)
                 const float2 a2 = make_float2(alpha, alpha);
@@ -772,7 +797,6 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 }
               }
             }
-            TR(5, nsub);
             // two columns per instruction; the bf16 pairs overwrite the low half of the registers
             const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
             float2 nm2[kG];
@@ -782,6 +806,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               nm2[g] = make_float2(a, a);
               acc[g][0] = acc[g][1] = make_float2(0.f, 0.f);
             }
+            racc[0] = racc[1] = make_float2(0.f, 0.f);
 #pragma unroll
             for (int c = 0; c < kW; c += 4) {
               if (C::kHasV && c == 32) ptx::tmem_wait_ld();  // (nothing is in flight on a second pass)
@@ -797,19 +822,29 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 x1.x = ptx::ex2_approx(x1.x);
                 x1.y = ptx::ex2_approx(x1.y);
               }
-              acc[c / kC][0] = ptx::add2(acc[c / kC][0], x0);
-              acc[c / kC][1] = ptx::add2(acc[c / kC][1], x1);
+              if (C::kWantMass) {
+                acc[c / kC][0] = ptx::add2(acc[c / kC][0], x0);
+                acc[c / kC][1] = ptx::add2(acc[c / kC][1], x1);
+              }
               if (C::kHasV) {
-                sr[c >> 1] = ptx::pack_bf16x2(x0.x, x0.y);
-                sr[(c >> 1) + 1] = ptx::pack_bf16x2(x1.x, x1.y);
+                const uint32_t u0 = ptx::pack_bf16x2(x0.x, x0.y), u1 = ptx::pack_bf16x2(x1.x, x1.y);
+                sr[c >> 1] = u0;
+                sr[(c >> 1) + 1] = u1;
+                racc[0] = ptx::add2(racc[0], ptx::unpack_bf16x2(u0));
+                racc[1] = ptx::add2(racc[1], ptx::unpack_bf16x2(u1));
               }
             }
-            TR(6, nsub);
             tsum = 0.f;
+            if (C::kWantMass) {
 #pragma unroll
-            for (int g = 0; g < kG; ++g) {
-              gsum[g] = (acc[g][0].x + acc[g][0].y) + (acc[g][1].x + acc[g][1].y);
-              tsum += gsum[g];
+              for (int g = 0; g < kG; ++g) {
+                gsum[g] = (acc[g][0].x + acc[g][0].y) + (acc[g][1].x + acc[g][1].y);
+                tsum += gsum[g];
+              }
+            }
+            if (C::kHasV) {
+              rsum = (racc[0].x + racc[0].y) + (racc[1].x + racc[1].y);
+              if (!C::kWantMass) tsum = rsum;
             }
             // after a pass with a fresh maximum every p is at most 2^8
             if (recentre || !__any_sync(0xffffffffu, !(tsum <= kSafeRowSum))) break;
@@ -821,6 +856,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
           }
           l += tsum;
+          if (C::kHasV && C::kWantMass) lr += rsum;
           if (C::kHasV) {
 #pragma unroll
             for (int c0 = 0; c0 < kW / 2; c0 += 32) ptx::tmem_st32(tSb + c0, &sr[c0]);
@@ -848,7 +884,6 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           ptx::tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&ctl->p_ready[qt]);
-          TR(7, nsub);
         }
         ++nsub;
       }
@@ -857,7 +892,8 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // ---- epilogue: O / l -> global
         if (T < p.nQt) {
           const bool valid = grow < p.N;
-          const float inv = (l > 0.f) ? 1.f / l : 0.f;
+          const float lo = C::kWantMass ? lr : l;
+          const float inv = (lo > 0.f) ? 1.f / lo : 0.f;
           const int64_t off = (int64_t)b * p.sb + (int64_t)h * p.sh + (int64_t)grow * p.sn;
           const int64_t pslot =
               ((((int64_t)(w - p.split_first) * p.split_parts + part) * 2 + qt) * 128 + row);
@@ -888,14 +924,14 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                                           __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
             } else if (valid) {
               if (p.o_f32) {
-                float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + off + c0);
+                float4* dst = reinterpret_cast<float4*>(static_cast<float*>(o_base) + off + c0);
 #pragma unroll
                 for (int c = 0; c < 32; c += 4)
                   dst[c >> 2] = make_float4(__uint_as_float(r[c]) * inv, __uint_as_float(r[c + 1]) * inv,
                                             __uint_as_float(r[c + 2]) * inv,
                                             __uint_as_float(r[c + 3]) * inv);
               } else {
-                uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.o) + off + c0);
+                uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(o_base) + off + c0);
 #pragma unroll
                 for (int c = 0; c < 32; c += 8) {
                   uint4 v;
@@ -1015,17 +1051,25 @@ __global__ void __launch_bounds__(32) build_tile_lists_kernel(const Params p) {
     part = r % parts;
     w = p.split_first + r / parts;
   }
-  const int bh = w / p.nPairs, pr = w % p.nPairs;
+  const int pbh = w / p.nPairs, pr = w % p.nPairs;
+  const int bh = pbh % (p.B * p.H);
+  const int32_t* offsets = p.offsets;
+  const int32_t* kv_idx = p.kv_idx;
+  if (p.problems != nullptr) {
+    const ProblemEntry* pe = p.problems + pbh / (p.B * p.H);
+    offsets = pe->offsets;
+    kv_idx = pe->kv_idx;
+  }
   const int W = (p.nKb + 31) >> 5;
   for (int i = lane; i < NB * W; i += 32) bm[i] = 0u;
   __syncwarp();
-  const int32_t nnz = __ldg(p.offsets + (int64_t)p.B * p.H * p.nQb);
+  const int32_t nnz = __ldg(offsets + (int64_t)p.B * p.H * p.nQb);
 #pragma unroll
   for (int n = 0; n < NB; ++n) {
     const int g = pr * NB + n;
     if (g >= p.nQb) continue;
     const int64_t row = (int64_t)bh * p.nQb + g;
-    const int32_t b = __ldg(p.offsets + row), e = __ldg(p.offsets + row + 1);
+    const int32_t b = __ldg(offsets + row), e = __ldg(offsets + row + 1);
     if (b < 0 || e < b || e > nnz || e - b > p.nKb) {
       report_error(p.status, LOSA_ERR_BAD_INDEX);
       continue;
@@ -1033,7 +1077,7 @@ __global__ void __launch_bounds__(32) build_tile_lists_kernel(const Params p) {
     const int b2 = b + (int)(((int64_t)(e - b) * part) / parts);
     const int e2 = b + (int)(((int64_t)(e - b) * (part + 1)) / parts);
     for (int i = b2 + lane; i < e2; i += 32) {
-      const int v = __ldg(p.kv_idx + i);
+      const int v = __ldg(kv_idx + i);
       if ((unsigned)v < (unsigned)p.nKb) atomicOr(&bm[n * W + (v >> 5)], 1u << (v & 31));
       else report_error(p.status, LOSA_ERR_BAD_INDEX);  // skipped, never used as an address
     }
@@ -1131,10 +1175,12 @@ template <int D>
 __global__ void __launch_bounds__(128) merge_parts_kernel(const Params p) {
   const int r = blockIdx.x, qt = blockIdx.y >> 3, chunk = blockIdx.y & 7;
   const int w = p.split_first + r;
-  const int bh = w / p.nPairs, pr = w % p.nPairs;
+  const int pbh = w / p.nPairs, pr = w % p.nPairs;
   const int T = 2 * pr + qt;
   if (T >= p.nQt) return;
+  const int bh = pbh % (p.B * p.H);
   const int b = bh / p.H, h = bh % p.H;
+  void* const o_base = (p.problems != nullptr) ? p.problems[pbh / (p.B * p.H)].o : p.o;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int parts = p.split_parts;
 #pragma unroll
@@ -1180,13 +1226,13 @@ __global__ void __launch_bounds__(128) merge_parts_kernel(const Params p) {
       }
       const int64_t off = (int64_t)b * p.sb + (int64_t)h * p.sh + (int64_t)grow * p.sn + d;
       if (p.o_f32) {
-        *reinterpret_cast<float4*>(static_cast<float*>(p.o) + off) =
+        *reinterpret_cast<float4*>(static_cast<float*>(o_base) + off) =
             make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
       } else {
         uint2 v;
         v.x = ptx::pack_bf16x2(acc.x * inv, acc.y * inv);
         v.y = ptx::pack_bf16x2(acc.z * inv, acc.w * inv);
-        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.o) + off) = v;
+        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(o_base) + off) = v;
       }
     }
   }
@@ -1234,18 +1280,8 @@ int make_map(CUtensorMap* m, const void* base, const Geometry& g, int box_rows) 
   return LOSA_OK;
 }
 
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
-  }
-  return n;
-}
-
 template <int D, int R, int C_, int MODE, int KT>
-int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Params prm,
+int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Params prm, int sms,
              cudaStream_t st) {
   using C = Cfg<D, R, C_, MODE, KT>;
   using Ctl = Control<C::kNK, C::kNV>;
@@ -1257,7 +1293,11 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
   const size_t smem =
       1024 + 2 * C::kQBytes + (size_t)(C::kNK + C::kNV) * C::kKVBytes + sizeof(Ctl);
   auto kern = losa_attn_kernel<D, R, C_, MODE, KT>;
-  static bool configured = false;
+  // (function attributes belong to a device: one flag per device ordinal)
+  static bool configured_on[kMaxDevices] = {};
+  int dev = 0;
+  LOSA_CUDA_TRY(cudaGetDevice(&dev));
+  bool& configured = configured_on[dev];
   if (!configured) {
     // the in-kernel register reallocation must fit the registers the CTA is launched with
     cudaFuncAttributes attr;
@@ -1269,8 +1309,6 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
     LOSA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     configured = true;
   }
-  int sms = sm_count();
-  if (sms <= 0) return LOSA_ERR_CUDA;
   const int ctas = min(sms, kMaxPersistentCtas);
   // The items of the last, partly filled wave of the persistent grid (all items, if there are
   // fewer than CTAs) are cut into parts of the key range, so that the wave ends after 1/parts of
@@ -1306,10 +1344,10 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
 
 template <int MODE>
 int dispatch(const Geometry& g, const void* q, const void* k, const void* v, const Params& prm,
-             cudaStream_t st) {
+             int sms, cudaStream_t st) {
   // K/V tiles of 128 keys everywhere (128 / C gathered key blocks, 128-wide MMAs)
 #define LOSA_CASE(d, r, c) \
-  if (g.D == d && g.R == r && g.C == c) return launch_t<d, r, c, MODE, 128>(g, q, k, v, prm, st)
+  if (g.D == d && g.R == r && g.C == c) return launch_t<d, r, c, MODE, 128>(g, q, k, v, prm, sms, st)
   LOSA_CASE(128, 128, 128);
   LOSA_CASE(64, 64, 64);
   LOSA_CASE(128, 128, 32);  // the paper's own block geometry
@@ -1324,30 +1362,35 @@ int dispatch(const Geometry& g, const void* q, const void* k, const void* v, con
 
 }  // namespace
 
-#ifdef LOSA_TRACE
-extern "C" int losa_debug_trace(void* host, size_t bytes) {
-  return (int)cudaMemcpyFromSymbol(host, g_trace, bytes < sizeof(g_trace) ? bytes : sizeof(g_trace));
-}
-#endif
 
 namespace {
 size_t part_o_bytes(const Geometry& g) {
   return (size_t)kMaxPersistentCtas * 2 * 128 * (size_t)g.D * sizeof(float);
 }
 // the last wave's items are cut into at most one unit per CTA
-int64_t max_units(const Geometry& g) { return (int64_t)g.B * g.H * g.nPairs + kMaxPersistentCtas; }
+int64_t max_units(const Geometry& g, int n_prob) {
+  return (int64_t)n_prob * g.B * g.H * g.nPairs + kMaxPersistentCtas;
+}
 int tile_list_cap(const Geometry& g) { return (g.nKb + 16 + 31) / 32 * 32; }  // union <= nKb, + padding of three sections
-size_t tl_count_bytes(const Geometry& g) { return ((size_t)max_units(g) * sizeof(int32_t) + 255) / 256 * 256; }
+size_t tl_count_bytes(const Geometry& g, int n_prob) {
+  return ((size_t)max_units(g, n_prob) * sizeof(int32_t) + 255) / 256 * 256;
+}
+size_t tl_entries_bytes(const Geometry& g, int n_prob) {
+  return ((size_t)max_units(g, n_prob) * tile_list_cap(g) * sizeof(uint32_t) + 255) / 256 * 256;
+}
 }  // namespace
 
-size_t attn_workspace_bytes(AttnMode mode, const Geometry& g) {
+void arm_stalled_launch(uint32_t polls) { g_stall_polls.store(polls); }
+
+size_t attn_workspace_bytes(AttnMode mode, const Geometry& g, int n_prob) {
   // attention output: counter, then one slot per partial unit (at most one per CTA) holding the
   // rows' (max, sum) and unnormalised O of both query tiles
   if (mode == kDense || mode == kSparse) {
     size_t bytes = kCounterBytes + kPartMlBytes + part_o_bytes(g);
     // sparse: the units' merged tile lists (count per unit, then tl_cap entries per unit)
-    if (mode == kSparse)
-      bytes += tl_count_bytes(g) + (size_t)max_units(g) * tile_list_cap(g) * sizeof(uint32_t);
+    if (mode == kSparse) bytes += tl_count_bytes(g, n_prob) + tl_entries_bytes(g, n_prob);
+    // batched launch: the table of the problems' tensor maps and pointers
+    if (n_prob > 1) bytes += (size_t)n_prob * sizeof(ProblemEntry);
     return bytes;
   }
   // counter, per-CTA row statistics, per-CTA table of one entry per row and key tile
@@ -1355,9 +1398,11 @@ size_t attn_workspace_bytes(AttnMode mode, const Geometry& g) {
          (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2);
 }
 
+// Batched launch (n_prob > 1, attention-only modes): `layers` is a host array of n_prob problems of
+// the geometry g; q, k, v, offsets, kv_idx and o are then ignored.
 int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, const void* v,
                 const int32_t* offsets, const int32_t* kv_idx, void* o, int o_dtype, float* mass,
-                float* lse, void* ws, cudaStream_t st) {
+                float* lse, void* ws, cudaStream_t st, int n_prob, const losa_layer_t* layers) {
   Params prm;
   prm.B = g.B;
   prm.H = g.H;
@@ -1366,8 +1411,11 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
   prm.nKb = g.nKb;
   prm.nQt = g.nQt;
   prm.nPairs = g.nPairs;
-  prm.nWork = g.B * g.H * g.nPairs;
-  if (prm.nWork > (int)kTlItemMask) return LOSA_ERR_UNSUPPORTED;  // the tile list's item headers hold 24 bits
+  if ((int64_t)n_prob * g.B * g.H * g.nPairs > (int64_t)kTlItemMask)
+    return LOSA_ERR_UNSUPPORTED;  // the tile list's item headers hold 24 bits
+  prm.nWork = n_prob * g.B * g.H * g.nPairs;
+  prm.nProb = n_prob;
+  prm.problems = nullptr;
   prm.offsets = offsets;
   prm.kv_idx = kv_idx;
   prm.o = o;
@@ -1387,18 +1435,46 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
   {
     char* tl = static_cast<char*>(ws) + kCounterBytes + kPartMlBytes + part_o_bytes(g);
     prm.tl_count = reinterpret_cast<int32_t*>(tl);
-    prm.tl_entries = reinterpret_cast<uint32_t*>(tl + tl_count_bytes(g));
+    prm.tl_entries = reinterpret_cast<uint32_t*>(tl + tl_count_bytes(g, n_prob));
     prm.tl_cap = tile_list_cap(g);
+    if (n_prob > 1) {
+      // the problems' table, behind the tile lists (dense mode has none), written before the launch
+      char* tab = tl + (mode == kSparse ? tl_count_bytes(g, n_prob) + tl_entries_bytes(g, n_prob) : 0);
+      std::vector<ProblemEntry> host(n_prob);
+      for (int i = 0; i < n_prob; ++i) {
+        int rc;
+        if ((rc = make_map(&host[i].map_q, layers[i].q, g, 128)) != LOSA_OK) return rc;
+        if ((rc = make_map(&host[i].map_k, layers[i].k, g, g.C)) != LOSA_OK) return rc;
+        if ((rc = make_map(&host[i].map_v, layers[i].v, g, g.C)) != LOSA_OK) return rc;
+        host[i].o = layers[i].o;
+        host[i].offsets = layers[i].offsets;
+        host[i].kv_idx = layers[i].kv_idx;
+      }
+      // (a copy from pageable memory is staged before the call returns: `host` may go out of scope)
+      LOSA_CUDA_TRY(cudaMemcpyAsync(tab, host.data(), (size_t)n_prob * sizeof(ProblemEntry),
+                                    cudaMemcpyHostToDevice, st));
+      prm.problems = reinterpret_cast<const ProblemEntry*>(tab);
+      q = layers[0].q;  // the kernel's parameter maps are unused but must be valid
+      k = layers[0].k;
+      v = layers[0].v;
+    }
   }
   prm.scale_log2 = g.scale * kLog2e;
-  prm.status = status_word_device();
-  if (!prm.status) return LOSA_ERR_CUDA;
+  int rc = LOSA_OK;
+  const DeviceState* dev = device_state(&rc);
+  if (!dev) return rc;
+  prm.status = dev->status_dev;
+  const int sms = dev->sm_count;
+  // one-shot diagnostic armed by losa_debug_stall_next_launch()
+  const uint32_t stall_polls = g_stall_polls.exchange(0u);
+  prm.stall = stall_polls > 0u ? 1 : 0;
+  prm.wait_polls = stall_polls > 0u ? stall_polls : ptx::kWaitPolls;
   LOSA_CUDA_TRY(cudaMemsetAsync(prm.work_counter, 0, sizeof(int), st));
   switch (mode) {
-    case kDense: return dispatch<kDense>(g, q, k, v, prm, st);
-    case kSparse: return dispatch<kSparse>(g, q, k, v, prm, st);
-    case kMass: return dispatch<kMass>(g, q, k, v, prm, st);
-    case kFused: return dispatch<kFused>(g, q, k, v, prm, st);
+    case kDense: return dispatch<kDense>(g, q, k, v, prm, sms, st);
+    case kSparse: return dispatch<kSparse>(g, q, k, v, prm, sms, st);
+    case kMass: return dispatch<kMass>(g, q, k, v, prm, sms, st);
+    case kFused: return dispatch<kFused>(g, q, k, v, prm, sms, st);
   }
   return LOSA_ERR_INVALID_ARG;
 }

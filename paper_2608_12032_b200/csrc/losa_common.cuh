@@ -12,10 +12,22 @@ namespace losa {
 // sized for it so that losa_workspace_bytes() needs no GPU.
 constexpr int kMaxPersistentCtas = 160;
 
-// Device-visible status word (pinned, mapped host memory).  Kernels record the first
-// error with a system-scope compare-and-swap; the host reads it after a stream sync.
-int* status_word_device();  // device pointer, valid on the current device
-int* status_word_host();
+// Per-device state of the library, created on a device's first call (thread-safe) and kept until
+// the process exits: the SM count and the device-visible status word (one int of pinned, mapped
+// host memory per device).  Kernels record the first error with a system-scope compare-and-swap;
+// the host reads the word after a stream sync.
+constexpr int kMaxDevices = 64;
+struct DeviceState {
+  int sm_count;
+  int* status_host;
+  int* status_dev;  // the same word as the kernels of this device address it
+};
+// State of the CURRENT device, or nullptr with *rc = LOSA_ERR_UNSUPPORTED (not an sm_100 GPU, or
+// a device ordinal beyond kMaxDevices) or LOSA_ERR_CUDA (a runtime call failed).
+const DeviceState* device_state(int* rc);
+// LOSA_OK if the current device can run the library's kernels (compute capability 10.x); makes no
+// allocation.
+int check_device();
 const char* set_cuda_error(cudaError_t e, const char* what);
 
 __device__ __forceinline__ void report_error(int* status, int code) {
@@ -48,8 +60,9 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 size_t select_workspace_bytes(int64_t rows, int nKb);
 int launch_select(int rows, int nKb, const float* mass, double tau, int fixed_count,
-                  int32_t* offsets, int32_t* kv_idx, int64_t kv_capacity, void* ws,
-                  cudaStream_t st);  // fixed_count > 0: keep that many blocks per row instead
+                  int32_t* offsets, int32_t* kv_idx, int64_t kv_capacity, void* ws, int* status,
+                  cudaStream_t st);  // fixed_count > 0: keep that many blocks per row instead;
+                                     // status: device-visible word that receives device-side errors
 int launch_row_recall(int rows, int nKb, const float* mass, const int32_t* offsets,
                       const int32_t* kv_idx, double* retained, double* total, cudaStream_t st);
 size_t select_noalloc_workspace_limit();
@@ -61,9 +74,11 @@ int launch_validate_csr(int rows, int nKb, const int32_t* offsets, const int32_t
 
 enum AttnMode { kDense = 0, kSparse = 1, kMass = 2, kFused = 3 };  // kFused: dense O and mass
 
-size_t attn_workspace_bytes(AttnMode mode, const Geometry& g);
+size_t attn_workspace_bytes(AttnMode mode, const Geometry& g, int n_prob = 1);
+void arm_stalled_launch(uint32_t polls);  // the next attention launch publishes no work (diagnostic)
 int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, const void* v,
                 const int32_t* offsets, const int32_t* kv_idx, void* o, int o_dtype, float* mass,
-                float* lse, void* ws, cudaStream_t st);
+                float* lse, void* ws, cudaStream_t st, int n_prob = 1,
+                const losa_layer_t* layers = nullptr);
 
 }  // namespace losa

@@ -48,16 +48,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: polls the barrier at most `kWaitPolls` times (with back-off sleeps once
-// the fast polls are used up, about a second in all) and also gives up as soon as another
-// thread of the CTA has raised `*abort_flag`.  Returns false when it gave up; the caller
-// then raises the flag itself and leaves its loop.  Nothing in this library spins forever.
+// Bounded wait: polls the barrier at most `limit` times (kWaitPolls in ordinary launches: with
+// the back-off sleeps that start once the fast polls are used up, about a second in all) and
+// also gives up as soon as another thread of the CTA has raised `*abort_flag`.  Returns false
+// when it gave up; the caller then raises the flag itself and leaves its loop.  Nothing in this
+// library spins forever.
 constexpr uint32_t kFastPolls = 1u << 14;
 constexpr uint32_t kWaitPolls = kFastPolls + (1u << 22);
 
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
-                                          volatile int* abort_flag) {
-  for (uint32_t it = 0; it < kWaitPolls; ++it) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t limit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (it >= kFastPolls) {
       if (*abort_flag) return false;
@@ -71,8 +72,8 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
 // scheduler): they sleep between polls from the start, so that their waiting costs neither issue
 // slots nor power that the softmax and MMA warps of the same SM could use.
 __device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity,
-                                                  volatile int* abort_flag) {
-  for (uint32_t it = 0; it < (1u << 22); ++it) {
+                                                  volatile int* abort_flag, uint32_t limit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (it >= 4) {
       if ((it & 1023u) == 0 && *abort_flag) return false;
@@ -96,33 +97,6 @@ __device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* m
       " [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(smem_u32(smem_dst)),
       "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w)
       : "memory");
-}
-
-// 4D tiled store shared -> global (rows outside the tensor are clipped by the hardware).
-__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, const void* smem_src, int x,
-                                             int y, int z, int w) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(
-          reinterpret_cast<uint64_t>(map)),
-      "r"(smem_u32(smem_src)), "r"(x), "r"(y), "r"(z), "r"(w)
-      : "memory");
-}
-
-__device__ __forceinline__ void tma_store_commit() {
-  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-
-__device__ __forceinline__ void tma_store_wait_read() {
-  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-}
-
-__device__ __forceinline__ void tma_store_wait_all() {
-  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-}
-
-// generic-proxy writes to shared memory -> visible to the async proxy (TMA store, MMA)
-__device__ __forceinline__ void fence_proxy_async_smem() {
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
 // ---------------------------------------------------------------- TMEM
@@ -189,38 +163,18 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
       : "memory");
 }
 
-// 16-column variant of tmem_st32.
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-      "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]),
-      "r"(r[15])
-      : "memory");
-}
-
 // ---------------------------------------------------------------- tcgen05.mma
 
-// Shared-memory matrix descriptor, 128-byte swizzle, bf16.
+// Shared-memory matrix descriptor, 128-byte swizzle, bf16, as its two 32-bit words.
+//   low word:  start address >> 4 (bits 13:0), leading byte offset >> 4 (bits 29:16)
+//   high word: stride byte offset >> 4 (bits 13:0), descriptor version 1 for sm_100 (bit 14),
+//              swizzle mode 2 = 128 bytes (bits 31:29)
 //   K-major operand  ([rows][64] slab, 128 B per row, 8-row swizzle atoms of 1024 B):
 //       lbo = 16 (unused for swizzled K-major), sbo = 1024
 //   MN-major operand (same slab read "transposed": 64 contiguous MN elements per K row):
 //       lbo = byte distance between 64-element MN groups, sbo = 1024 (8 K rows)
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo_bytes,
-                                                    uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
-  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
-  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
-  d |= (uint64_t)1 << 46;  // descriptor version for sm_100
-  d |= (uint64_t)2 << 61;  // 128-byte swizzle
-  return d;
-}
-
-// The same descriptor split into its two 32-bit words, so that the issuing thread only adds a
-// pre-shifted byte offset to the low word per MMA (the address field cannot carry: shared-memory
-// addresses are below 256 KiB).
+// The issuing thread only adds a pre-shifted byte offset to the low word per MMA (the address
+// field cannot carry: shared-memory addresses are below 256 KiB).
 __host__ __device__ constexpr uint32_t smem_desc_hi_sw128(uint32_t sbo_bytes) {
   return ((sbo_bytes >> 4) & 0x3FFF) | (1u << 14) | (2u << 29);
 }
@@ -239,64 +193,9 @@ __host__ __device__ constexpr uint32_t idesc_bf16_f32(int M, int N, bool a_mn_ma
          | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
-                                       uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t"
-      ".reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
-      "}" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
-                                       uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t"
-      ".reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t"
-      "}" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
-// Same two forms with the descriptors given as (low word, shared high word).
-__device__ __forceinline__ void mma_ss_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo,
-                                            uint32_t hi, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t"
-      ".reg .pred p;\n\t"
-      ".reg .b64 da, db;\n\t"
-      "setp.ne.b32 p, %5, 0;\n\t"
-      "mov.b64 da, {%1, %3};\n\t"
-      "mov.b64 db, {%2, %3};\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t"
-      "}" ::"r"(d_tmem),
-      "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
-__device__ __forceinline__ void mma_ts_lohi(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo,
-                                            uint32_t hi, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t"
-      ".reg .pred p;\n\t"
-      ".reg .b64 db;\n\t"
-      "setp.ne.b32 p, %5, 0;\n\t"
-      "mov.b64 db, {%2, %3};\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t"
-      "}" ::"r"(d_tmem),
-      "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
-// Forms that take ready-made 64-bit descriptors, so that nothing but the MMA itself has to be
-// issued between two MMAs (the descriptors are built while the issuer waits for its operands).
+// D[tmem] (+)= A * B with A from shared memory (mma_ss_*) or from TMEM (mma_ts_*), B from shared
+// memory.  Forms that take ready-made 64-bit descriptors, so that nothing but the MMA itself has to
+// be issued between two MMAs (the descriptors are built while the issuer waits for its operands).
 __device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) {
   uint64_t d;
   asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
@@ -370,6 +269,11 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return r;
 }
 
+// The two bf16 values of a packed pair, widened to fp32 (exact).
+__device__ __forceinline__ float2 unpack_bf16x2(uint32_t u) {
+  return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+}
+
 // Packed fp32 pairs (one instruction, two lanes of the FMA pipe).
 __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
   float2 d;
@@ -429,10 +333,13 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // 2^x for a pair on the FMA pipe instead of the special-function unit: round x to the nearest
 // integer n with the 1.5 * 2^23 trick, evaluate a quintic for 2^(x - n) on [-0.5, 0.5] (maximum
 // relative error 2.4e-7 in fp32, the same as ex2.approx) and add n to the exponent field.
-// Inputs below -127 (masked keys hold -inf) are clamped and come out as zero or a denormal.
+// Inputs below -127 (masked keys hold -inf) are clamped and come out as zero or a denormal;
+// inputs above 127 are clamped too and come out as 2^127, far beyond the row-sum range the
+// callers accept, so that an overflow shows in the sum instead of wrapping into the sign bit.
+// (NaN also clamps to a finite value: callers that must see NaN look at the other columns.)
 __device__ __forceinline__ float2 ex2_poly2(float2 x) {
-  x.x = fmaxf(x.x, -127.f);
-  x.y = fmaxf(x.y, -127.f);
+  x.x = fminf(fmaxf(x.x, -127.f), 127.f);
+  x.y = fminf(fmaxf(x.y, -127.f), 127.f);
   const float2 t = add2(x, make_float2(12582912.f, 12582912.f));
   const float2 n = add2(t, make_float2(-12582912.f, -12582912.f));
   const float2 f = add2(x, make_float2(-n.x, -n.y));

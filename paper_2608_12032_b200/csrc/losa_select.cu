@@ -5,7 +5,7 @@
 //                           registers, the threshold value found bit by bit with masked
 //                           fixed-point sums (no sort); the kept set is written as a bitmap
 //                           over block indices plus its size.
-//      select_rows_kernel   longer rows (and the no-allocation entry point): one CTA per
+//      select_rows_kernel   longer rows: one CTA per
 //                           row, sort (mass descending, index ascending) as 64-bit integer
 //                           keys in shared memory, fp64 prefix sum along the sorted order,
 //                           shortest prefix reaching tau; same outputs.
@@ -35,6 +35,7 @@ select_rows_kernel(const float* __restrict__ mass, int nKb, int n2, double tau, 
   uint32_t* bitmap = reinterpret_cast<uint32_t*>(keys + n2);
   __shared__ double warp_total[kSelThreads / 32];
   __shared__ int first_pos;
+  __shared__ double row_total;
 
   const int tid = threadIdx.x;
   const int64_t row = blockIdx.x;
@@ -46,7 +47,7 @@ select_rows_kernel(const float* __restrict__ mass, int nKb, int n2, double tau, 
     unsigned long long key = kPadKey;
     if (i < nKb) {
       float m = mrow[i];
-      if (!(m >= 0.0f)) {  // negative or NaN
+      if (!(m >= 0.0f) || m > 8.0f) {  // negative, NaN, or far beyond any mass
         bad = true;
         m = 0.0f;
       }
@@ -103,9 +104,16 @@ select_rows_kernel(const float* __restrict__ mass, int nKb, int n2, double tau, 
       break;
     }
   }
+  if (tid == kSelThreads - 1) row_total = base + incl;
   __syncthreads();
   int s = first_pos;
   if (tau >= 1.0 || s > nKb) s = nKb;
+  // same rule as the warp-per-row kernel: a row whose masses add up to more than 8 is reported and
+  // keeps every block
+  if (row_total > 8.0) {
+    s = nKb;
+    if (tid == 0) report_error(status, LOSA_ERR_BAD_MASS);
+  }
   if (fixed_count > 0) s = min(fixed_count, nKb);  // fixed-ratio rule: the k heaviest blocks
 
   for (int i = lo; i < hi; ++i) {
@@ -139,6 +147,7 @@ select_rows_warp_kernel(const float* __restrict__ mass, int rows, int nKb, doubl
   uint32_t bits[K];
   unsigned long long fx[K];
   bool bad = false;
+  float row_sum = 0.0f;
 #pragma unroll
   for (int k = 0; k < K; ++k) {
     const int i = k * 32 + lane;
@@ -152,6 +161,16 @@ select_rows_warp_kernel(const float* __restrict__ mass, int rows, int nKb, doubl
     // block for the fixed-ratio rule, which counts; blocks past the row's end weigh nothing
     if (fixed_count > 0) fx[k] = (i < nKb) ? 1ull : 0ull;
     else fx[k] = (unsigned long long)((double)m * 1152921504606846976.0);
+    row_sum += m;
+  }
+  // The fixed-point sums below hold at most 16: a row whose masses add up to more than 8 (a mass
+  // row sums to 1) is reported, and keeps every block, instead of wrapping silently.
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) row_sum += __shfl_xor_sync(0xffffffffu, row_sum, d);
+  if (fixed_count <= 0 && row_sum > 8.0f) {
+    bad = true;
+#pragma unroll
+    for (int k = 0; k < K; ++k) fx[k] = 0ull;
   }
   if (__any_sync(0xffffffffu, bad) && lane == 0) report_error(status, LOSA_ERR_BAD_MASS);
 
@@ -352,10 +371,8 @@ size_t select_workspace_bytes(int64_t rows, int nKb) {
 }
 
 int launch_select(int rows, int nKb, const float* mass, double tau, int fixed_count,
-                  int32_t* offsets, int32_t* kv_idx, int64_t kv_capacity, void* ws,
+                  int32_t* offsets, int32_t* kv_idx, int64_t kv_capacity, void* ws, int* status,
                   cudaStream_t st) {
-  int* status = status_word_device();
-  if (!status) return LOSA_ERR_CUDA;
   int32_t* counts = static_cast<int32_t*>(ws);
   uint32_t* bitmaps = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) +
                                                   align_up((size_t)rows * sizeof(int32_t), 256));
@@ -372,6 +389,7 @@ int launch_select(int rows, int nKb, const float* mass, double tau, int fixed_co
     const int n2 = next_pow2(nKb);
     const int words = (nKb + 31) / 32;
     const size_t smem = (size_t)n2 * 8 + (size_t)words * 4;
+    // (a function attribute belongs to the current device: set on every call, it costs nothing)
     if (smem > 48 * 1024) {
       LOSA_CUDA_TRY(cudaFuncSetAttribute(select_rows_kernel,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -395,7 +413,6 @@ constexpr size_t kStaticStatusBytes = 256;
 static __device__ __align__(256) unsigned char g_select_scratch[LOSA_SELECT_NOALLOC_MAX_SCRATCH];
 
 namespace {
-constexpr int kMaxDevices = 64;
 unsigned char* g_scratch_addr[kMaxDevices] = {};  // device address of g_select_scratch, per device
 }  // namespace
 
@@ -422,23 +439,9 @@ int launch_select_noalloc(int rows, int nKb, const float* mass, double tau, int3
   // the array keeps the previous call's contents: the status word must start at zero; counts
   // and bitmaps are fully rewritten by the first kernel before anything reads them
   LOSA_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int), st));
-  int32_t* counts = reinterpret_cast<int32_t*>(ws);
-  uint32_t* bitmaps =
-      reinterpret_cast<uint32_t*>(ws + align_up((size_t)rows * sizeof(int32_t), 256));
-  const int n2 = next_pow2(nKb);
-  const int words = (nKb + 31) / 32;
-  const size_t smem = (size_t)n2 * 8 + (size_t)words * 4;
-  if (smem > 48 * 1024) {
-    LOSA_CUDA_TRY(cudaFuncSetAttribute(select_rows_kernel,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  }
-  select_rows_kernel<<<rows, kSelThreads, smem, st>>>(mass, nKb, n2, tau, 0, counts, bitmaps,
-                                                      status);
-  scan_counts_kernel<<<1, 1024, 0, st>>>(counts, rows, offsets, kv_capacity, status);
-  const int warps_per_cta = 8;
-  expand_rows_kernel<<<(rows + warps_per_cta - 1) / warps_per_cta, warps_per_cta * 32, 0, st>>>(
-      bitmaps, offsets, rows, nKb, kv_idx, kv_capacity);
-  LOSA_CUDA_TRY(cudaGetLastError());
+  // the same kernels, dispatch and workspace layout as losa_select
+  const int rc = launch_select(rows, nKb, mass, tau, 0, offsets, kv_idx, kv_capacity, ws, status, st);
+  if (rc != LOSA_OK) return rc;
   if (device_status)
     LOSA_CUDA_TRY(cudaMemcpyAsync(device_status, status, sizeof(int), cudaMemcpyDeviceToDevice, st));
   return LOSA_OK;
@@ -446,8 +449,10 @@ int launch_select_noalloc(int rows, int nKb, const float* mass, double tau, int3
 
 int launch_row_recall(int rows, int nKb, const float* mass, const int32_t* offsets,
                       const int32_t* kv_idx, double* retained, double* total, cudaStream_t st) {
-  int* status = status_word_device();
-  if (!status) return LOSA_ERR_CUDA;
+  int rc = LOSA_OK;
+  const DeviceState* dev = device_state(&rc);
+  if (!dev) return rc;
+  int* status = dev->status_dev;
   row_recall_kernel<<<(rows + 7) / 8, 256, 0, st>>>(mass, rows, nKb, offsets, kv_idx, retained,
                                                     total, status);
   LOSA_CUDA_TRY(cudaGetLastError());
@@ -456,8 +461,10 @@ int launch_row_recall(int rows, int nKb, const float* mass, const int32_t* offse
 
 int launch_validate_csr(int rows, int nKb, const int32_t* offsets, const int32_t* kv_idx,
                         cudaStream_t st) {
-  int* status = status_word_device();
-  if (!status) return LOSA_ERR_CUDA;
+  int rc = LOSA_OK;
+  const DeviceState* dev = device_state(&rc);
+  if (!dev) return rc;
+  int* status = dev->status_dev;
   validate_csr_kernel<<<(rows + 7) / 8, 256, 0, st>>>(rows, nKb, offsets, kv_idx, status);
   LOSA_CUDA_TRY(cudaGetLastError());
   return LOSA_OK;

@@ -1,0 +1,111 @@
+"""losa_sparse_attn_batched: several problems (layers, requests) of one shape, each with its own
+tensors and its own frozen pattern, in one persistent launch, against the single calls and the
+fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import losa_oracle as orc
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+def lib():
+    import paper_2608_12032_b200 as losa
+    return losa
+
+
+def make_layers(L, B, H, N, D, R, C, seed):
+    nQb, nKb = -(-N // R), -(-N // C)
+    host, dev = [], []
+    for l in range(L):
+        q = util.rand_bf16((B, H, N, D), seed + 10 * l, 1.5)
+        k = util.rand_bf16((B, H, N, D), seed + 10 * l + 1, 1.5)
+        v = util.rand_bf16((B, H, N, D), seed + 10 * l + 2)
+        # every layer its own pattern, with a different density
+        off, idx = util.random_csr(B * H * nQb, nKb, seed + l, (0.2, 0.5, 0.8, 0.35)[l % 4])
+        host.append((q, k, v, off, idx))
+        dev.append((q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(off).cuda(), torch.from_numpy(idx).cuda()))
+    return host, dev
+
+
+def items(B, H, N):
+    return B * H * ((-(-N // 128) + 1) // 2)
+
+
+def cut_into_parts(n_items):
+    """The library's host rule, restated: are the work items of the last wave cut into parts?"""
+    ctas = min(torch.cuda.get_device_properties(0).multi_processor_count, 160)
+    rest = n_items if n_items < ctas else n_items % ctas
+    return rest > 0 and ctas // rest >= 2
+
+
+@pytest.mark.parametrize("B,H,N,D,R,C", [(1, 5, 128 * 31 + 70, 64, 64, 64), (1, 5, 128 * 32 - 9, 128, 128, 32)])
+def test_three_layers_in_one_launch_equal_the_single_calls_bit_for_bit(B, H, N, D, R, C):
+    losa = lib()
+    L = 3
+    if cut_into_parts(items(B, H, N)) or cut_into_parts(L * items(B, H, N)):
+        pytest.skip("this GPU's SM count cuts the last wave into parts for this shape")
+    host, dev = make_layers(L, B, H, N, D, R, C, 300)
+    outs = losa.losa_sparse_attn_batched(dev, R, C, out_dtype=torch.float32)
+    assert losa.losa_async_status() == 0
+    for l, (q, k, v, off, idx) in enumerate(dev):
+        single = losa.losa_sparse_attn(q, k, v, off, idx, R, C, out_dtype=torch.float32)
+        assert losa.losa_async_status() == 0
+        assert torch.equal(outs[l], single), f"layer {l}"
+    # and against the oracle, layer by layer, on a sample of query blocks
+    nQb = -(-N // R)
+    ids = np.array(sorted({0, 1, nQb - 1, nQb, 2 * nQb + 3, B * H * nQb - 1, B * H * nQb - 2}), dtype=np.int32)
+    for l, (q, k, v, off, idx) in enumerate(host):
+        ref = orc.sparse_attn(util.to_np(q), util.to_np(k), util.to_np(v), R, C, off, idx, row_ids=ids)
+        got = np.zeros_like(ref)
+        flat = outs[l].reshape(B * H, N, D).cpu().numpy()
+        for n, r in enumerate(ids):
+            bh, i = divmod(int(r), nQb)
+            blk = flat[bh, i * R:(i + 1) * R]
+            got[n, : blk.shape[0]] = blk
+        d = np.abs(got - ref)
+        assert d.max() <= util.MAX_ABS_TOL and d.mean() <= util.MEAN_ABS_TOL, (l, d.max(), d.mean())
+
+
+@pytest.mark.parametrize("L", [1, 2, 7])
+def test_small_layers_batched_match_the_oracle(L):
+    """Layers of the Small workload's size (32 work items each): alone each is cut into parts and
+    merged, batched they may not be.  A part exponentiates against its own reference, so its bf16
+    weights round differently: the single and the batched call are two approximations of the same
+    values, each compared with the oracle element by element."""
+    losa = lib()
+    B, H, N, D, R, C = 1, 4, 2048 - 30, 64, 64, 64
+    host, dev = make_layers(L, B, H, N, D, R, C, 500)
+    outs = losa.losa_sparse_attn_batched(dev, R, C, out_dtype=torch.float32)
+    outs16 = losa.losa_sparse_attn_batched(dev, R, C, out_dtype=torch.bfloat16)
+    assert losa.losa_async_status() == 0
+    for l, (q, k, v, off, idx) in enumerate(host):
+        ref = orc.blocks_to_tokens(
+            orc.sparse_attn(util.to_np(q), util.to_np(k), util.to_np(v), R, C, off, idx), B, H, N)
+        util.assert_output_close(outs[l], ref, f"layer {l} of {L}")
+        assert torch.equal(outs16[l], outs[l].bfloat16())
+        single = losa.losa_sparse_attn(*dev[l], R, C, out_dtype=torch.float32)
+        assert losa.losa_async_status() == 0
+        util.assert_output_close(single, ref, f"layer {l} alone")
+        assert (single - outs[l]).abs().max().item() <= util.MAX_ABS_TOL
+
+
+def test_batched_call_reports_a_bad_index_of_one_layer_and_checks_its_arguments():
+    losa = lib()
+    B, H, N, D, R, C = 1, 2, 900, 64, 64, 64
+    host, dev = make_layers(2, B, H, N, D, R, C, 700)
+    bad = host[1][4].copy()
+    bad[3] = 1000
+    dev[1] = dev[1][:4] + (torch.from_numpy(bad).cuda(),)
+    outs = losa.losa_sparse_attn_batched(dev, R, C, out_dtype=torch.float32)
+    assert losa.losa_status_string(losa.losa_async_status()) == "LOSA_ERR_BAD_INDEX"
+    assert all(torch.isfinite(o).all() for o in outs)
+    # the other layer is unaffected
+    ref = losa.losa_sparse_attn(*dev[0], R, C, out_dtype=torch.float32)
+    assert losa.losa_async_status() == 0
+    assert (ref - outs[0]).abs().max().item() <= util.MAX_ABS_TOL
+    with pytest.raises(losa.LosaError) as e:
+        losa.losa_sparse_attn_batched(dev, R, C, ws=torch.empty(1024, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == -3

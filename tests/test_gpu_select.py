@@ -114,6 +114,26 @@ def test_select_flags_negative_and_nan_mass():
     assert losa.losa_status_string(run[2]) == "LOSA_ERR_BAD_MASS"
 
 
+@pytest.mark.parametrize("nKb", [40, 1500])
+def test_select_flags_rows_whose_masses_do_not_look_like_masses(nKb):
+    """Masses above 8, and rows whose masses add up to more than 8 (beyond the warp kernel's
+    fixed-point range), are reported instead of giving a silently wrong pattern; a row with a bad
+    sum keeps every block.  Both selection kernels (nKb = 1500 takes the sorting one)."""
+    losa = lib()
+    m = random_mass(4, nKb, 11)
+    m[2] = 1.0            # each value passes, the row adds up to nKb
+    off, idx, status = run_select(m, 0.9)
+    assert losa.losa_status_string(status) == "LOSA_ERR_BAD_MASS"
+    assert off[3] - off[2] == nKb
+    sel = orc.select(m.astype(np.float64), 0.9)
+    rows = util.csr_rows(off, idx[: off[-1]])
+    ref = util.csr_rows(sel.offsets, sel.kv_idx)
+    assert [rows[r] for r in (0, 1, 3)] == [ref[r] for r in (0, 1, 3)]  # the other rows are untouched
+    m = random_mass(4, nKb, 12)
+    m[1, 7] = 9.0
+    assert losa.losa_status_string(run_select(m, 0.9)[2]) == "LOSA_ERR_BAD_MASS"
+
+
 def test_select_host_side_argument_errors():
     losa = lib()
     mass = torch.rand(1, 1, 4, 8, device="cuda")
@@ -124,6 +144,11 @@ def test_select_host_side_argument_errors():
     with pytest.raises(losa.LosaError) as e:
         losa.losa_select(mass, 0.9, ws=torch.empty(16, dtype=torch.uint8, device="cuda"))
     assert e.value.code == -3
+    # rows longer than LOSA_SELECT_MAX_KEY_BLOCKS are refused before any launch
+    long_rows = torch.zeros(1, 1, 1, 8193, device="cuda")
+    with pytest.raises(losa.LosaError) as e:
+        losa.losa_select(long_rows, 0.9)
+    assert e.value.code == -2
 
 
 @pytest.mark.parametrize("rows,nKb,k", [(16, 33, 1), (16, 33, 20), (8, 256, 170), (4, 929, 557), (8, 40, 40)])
