@@ -43,13 +43,30 @@ namespace {
 
 std::atomic<uint32_t> g_stall_polls{0u};  // > 0: the next attention launch is a diagnostic one
 
-constexpr int kThreads = 384;  // 2 softmax warpgroups + 1 utility warpgroup (TMA, 2 MMA issuers, scheduler)
-constexpr int kRegsSoftmax = 216, kRegsUtility = 72, kRegsAtLaunch = 168;
-// setmaxnreg only moves registers inside the CTA's launch allocation: the increase waits until
-// the decrease has released enough, so the totals must balance or the increase never returns.
-static_assert(128 * kRegsUtility + 256 * kRegsSoftmax <= kThreads * kRegsAtLaunch,
-              "register reallocation exceeds the CTA's launch allocation");
-static_assert(kThreads * kRegsAtLaunch <= 65536, "launch allocation exceeds the register file");
+// Thread layout.  Warps 0-3 are the utility warpgroup (TMA, 2 MMA issuers, scheduler); the softmax
+// warps follow.  Two layouts:
+//   one thread per query row (SPLIT = false): 2 softmax warpgroups, one per query tile, each thread
+//     holding a whole 128-column S row.  Used by the mass pass and the fused construction step,
+//     and as the fallback of the attention-only modes.
+//   two threads per query row (SPLIT = true): 4 softmax warpgroups, two per query tile, each
+//     thread holding 64 columns.  A warp's ex2 instructions occupy it for 8 issue cycles each and
+//     its other instructions do not overlap them (measured on the loop alone: 1301 cycles per
+//     128-column row with one warp per scheduler partition, 1130 with two), so a query tile's
+//     softmax needs two warps per partition to keep the special-function unit busy; the two warps
+//     never talk to each other on the common path (see the softmax role).
+template <bool SPLIT>
+struct Lay {
+  static constexpr int kSoftmaxWarps = SPLIT ? 16 : 8;
+  static constexpr int kThreads = 128 + 32 * kSoftmaxWarps;
+  static constexpr int kRegsSoftmax = SPLIT ? 104 : 216;
+  static constexpr int kRegsUtility = SPLIT ? 64 : 72;
+  static constexpr int kRegsAtLaunch = SPLIT ? 96 : 168;
+  // setmaxnreg only moves registers inside the CTA's launch allocation: the increase waits until
+  // the decrease has released enough, so the totals must balance or the increase never returns.
+  static_assert(128 * kRegsUtility + 32 * kSoftmaxWarps * kRegsSoftmax <= kThreads * kRegsAtLaunch,
+                "register reallocation exceeds the CTA's launch allocation");
+  static_assert(kThreads * kRegsAtLaunch <= 65536, "launch allocation exceeds the register file");
+};
 // The utility warps take the LOWEST warp ids.  When several warps of a scheduler partition are
 // ready, the hardware favours the lower (older) ids; a softmax warp in an arithmetic-dense
 // stretch is ready every cycle, and with the MMA issuer behind it in that order each of the
@@ -61,7 +78,7 @@ constexpr int kTmemCols = 512;
 constexpr size_t kCounterBytes = 256;  // head of the workspace: the work-item counter
 constexpr size_t kRowstatBytes = (size_t)kMaxPersistentCtas * 2 * 128 * sizeof(float2);
 constexpr size_t kPartMlBytes = kRowstatBytes;  // same shape: [slot][2][128] float2
-constexpr int kTlChunks = 8;
+constexpr int kTlChunks = 4;
 constexpr uint32_t kTlItem = 1u << 28, kTlEnd = 2u << 28;  // entry type in bits 31:28 (0 = tile)
 // An item header carries the work item in bits 23:0 and, for a unit that covers only part of the
 // item's key range, the part index in bits 26:24 and a flag in bit 27.
@@ -75,6 +92,8 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;
 constexpr float kSafeRowSum = 1.099511627776e12f;  // 2^40: a tile's row sum beyond this re-centres the reference
+// two threads per row: a tile's half-row sum beyond 2^60 (or NaN) sends the work unit to the fallback
+constexpr float kSplitSafeSum = 1.152921504606846976e18f;
 
 template <int D, int R, int C_, int MODE, int KT>
 struct Cfg {
@@ -145,11 +164,16 @@ struct Params {
   float2* table;  // mass modes: [grid][2][nKb][128] (sum of p, reference max) per row and key tile
   float scale_log2;
   int* status;
+  // Work units whose scores outgrew the fixed reference of the two-threads-per-row kernel: it
+  // appends them here, and a second launch (one thread per row, moving reference) recomputes them.
+  int* redo_count;
+  int* redo_list;
+  int redo;             // this launch processes redo_list[0 .. *redo_count) instead of all units
   uint32_t wait_polls;  // bound of every device-side wait, in polls (ptx::kWaitPolls)
   int stall;            // diagnostic launch: the scheduler publishes nothing, so that every wait runs out
 };
 
-template <int NK, int NV>
+template <int NK, int NV, bool SPLIT>
 struct Control {
   uint64_t q_full[2], q_empty[2];
   uint64_t k_full[NK], k_empty[NK];
@@ -164,6 +188,12 @@ struct Control {
   uint32_t tmem_base;
   uint32_t mma_lock;  // held while a burst of MMAs is issued
   int abort_flag;
+  // two threads per row: the pair's barrier per (query tile, lane quarter), the row sums the second
+  // half hands to the first at the end of an item (two sets, used in turn), and the last work unit
+  // this CTA sent to the fallback
+  uint64_t pair_bar[SPLIT ? 8 : 1];
+  float xch[SPLIT ? 2 * 2 * 128 : 1];
+  int ovf_unit;
 };
 
 #define LOSA_WAIT_RELAXED(bar, parity)                                   \
@@ -243,12 +273,14 @@ struct Control {
     ++te;                                                                            \
   } while (0)
 
-template <int D, int R, int C_, int MODE, int KT>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int D, int R, int C_, int MODE, int KT, bool SPLIT>
+__global__ void __launch_bounds__(Lay<SPLIT>::kThreads, 1)
 losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, const Params p) {
   using C = Cfg<D, R, C_, MODE, KT>;
-  using Ctl = Control<C::kNK, C::kNV>;
+  using L = Lay<SPLIT>;
+  using Ctl = Control<C::kNK, C::kNV, SPLIT>;
+  static_assert(!SPLIT || (C::kHasV && !C::kWantMass), "two threads per row: attention-only modes");
   constexpr int kC = C::kC, kG = C::kG, kQBT = C::kQBT, kNB = C::kNB, kW = C::kW, kNS = C::kNS;
   constexpr uint32_t kSStride = C::kSStride, kNVs = C::kNV > 0 ? C::kNV : 1;
   constexpr uint32_t kQMask = (1u << kQBT) - 1u;
@@ -259,9 +291,15 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   // wait on the chain of their steps, not on that unit (tried twice, slower each time).
   constexpr int kPolyEvery = (MODE == kMass) ? 4 : 0;
 
-  extern __shared__ uint8_t smem_raw[];
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  // (the swizzled tiles need 1024-byte alignment; the one-thread-per-row layout has room for the
+  // slack, the other relies on the declared alignment and checks it)
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
+  if (SPLIT && smem != smem_raw) {
+    if (threadIdx.x == 0) report_error(p.status, LOSA_ERR_CUDA);
+    return;
+  }
   uint8_t* sQ = smem;
   uint8_t* sK = sQ + 2 * C::kQBytes;
   uint8_t* sV = sK + C::kNK * C::kKVBytes;
@@ -277,9 +315,9 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         ptx::mbar_init(&ctl->s_full[i][u], 1);
         ptx::mbar_init(&ctl->s_free[i][u], 4);  // one elected arrival per softmax warp
       }
-      ptx::mbar_init(&ctl->p_ready[i], 4);  // one elected arrival per softmax warp
+      ptx::mbar_init(&ctl->p_ready[i], L::kSoftmaxWarps / 2);  // one elected arrival per softmax warp
       ptx::mbar_init(&ctl->o_done[i], 1);
-      ptx::mbar_init(&ctl->o_free[i], 128);
+      ptx::mbar_init(&ctl->o_free[i], 128);  // the threads that read O out
       ptx::mbar_init(&ctl->wg_bar[i], 128);
     }
     for (int i = 0; i < C::kNK; ++i) {
@@ -292,8 +330,12 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
     for (int i = 0; i < kTlChunks; ++i) {
       ptx::mbar_init(&ctl->tl_full[i], 1);
-      // readers of the tile list: producer, 2 MMA issuers, 8 softmax warps
-      ptx::mbar_init(&ctl->tl_empty[i], 11);
+      // readers of the tile list: producer, 2 MMA issuers, the softmax warps
+      ptx::mbar_init(&ctl->tl_empty[i], 3 + L::kSoftmaxWarps);
+    }
+    if (SPLIT) {
+      for (int i = 0; i < 8; ++i) ptx::mbar_init(&ctl->pair_bar[i], 2);
+      ctl->ovf_unit = -1;
     }
     ptx::mbar_init(&ctl->drain, 2);  // the MMA issuers arrive on the abort path
     ctl->mma_lock = 0;
@@ -317,7 +359,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   // The softmax warpgroups hold a whole S row per thread: the utility warpgroup gives registers
   // up and the softmax warpgroups take them.
   if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsUtility));
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(L::kRegsUtility));
   if (warp == kProducerWarp) {
     // ------------------------------------------------------------------ TMA producer
     // (the whole warp walks the tile list; lane 0 alone issues the copies)
@@ -508,10 +550,13 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               if (C::kHasV && pend) {
                 // O += P V for the previous key tile of this query tile
                 if (kLoDesc) {
+                  // (two threads per row: each half packs its P over the head of its own 64 score
+                  // columns, so the second half of the keys reads its operand from column 64 on)
                   ptx::mma_ts_lo(tO, tS, vd[0], kDescHi, C::kIdescPV, pv_item > 0 ? 1u : 0u);
 #pragma unroll
                   for (int kk = 1; kk < kW / 16; ++kk)
-                    ptx::mma_ts_lo(tO, tS + kk * 8, vd[kk], kDescHi, C::kIdescPV, 1u);
+                    ptx::mma_ts_lo(tO, tS + (SPLIT ? (kk & 3) * 8 + (kk >> 2) * 64 : kk * 8), vd[kk],
+                                   kDescHi, C::kIdescPV, 1u);
                 } else {
                   ptx::mma_ts_d(tO, tS, vd64[0], C::kIdescPV, pv_item > 0 ? 1u : 0u);
 #pragma unroll
@@ -588,7 +633,11 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       // work items are drawn from a global counter, in head-major order, so that a CTA that
       // finishes early takes the next item instead of idling at the end of the launch
       int w = 0;
-      if (lane == 0) w = atomicAdd(p.work_counter, 1);
+      if (lane == 0) {
+        w = atomicAdd(p.work_counter, 1);
+        // fallback launch: the units the two-threads-per-row kernel could not finish
+        if (p.redo) w = (w < *p.redo_count) ? p.redo_list[w] : p.nUnits;
+      }
       w = __shfl_sync(0xffffffffu, w, 0);
       if (w >= p.nUnits) break;
       // units past split_first are parts of the key range of the last items
@@ -641,9 +690,9 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
     }
   }
-  } else {
+  } else if constexpr (!SPLIT) {
     // ------------------------------------------------------------------ softmax warpgroups
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(L::kRegsSoftmax));
     const int qt = (warp >> 2) - 1, wl = warp & 3;  // TMEM lanes 32 * (warp % 4) .. + 31
     const int row = wl * 32 + lane;
     const uint32_t lane_base = (uint32_t)(wl * 32) << 16;
@@ -999,6 +1048,245 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         ++nwg;
       }
     }
+  } else {
+    // ------------------------------------------------------------------ softmax warps, two per row
+    // Warps 4-11 serve query tile 0, warps 12-19 query tile 1; within a query tile the first
+    // four warps (half 0) take key columns 0-63 of every S, the other four (half 1) columns
+    // 64-127, each thread 64 columns of its row.  A pair of warps (same rows, the two halves)
+    // shares a scheduler partition, so one warp's packing and summing fills the issue slots the
+    // other's ex2 leaves empty.  On the common path the two never synchronise:
+    //   * the reference the exponentials are taken against is the row maximum of the item's first
+    //     tile, which each half computes for itself over all 128 columns, and it never moves;
+    //   * each half packs its P over the head of its own score columns and keeps its own sum;
+    //   * if a half's sum of a tile leaves the safe range (scores that rose 40 nats above the
+    //     first tile), the whole work unit is handed to the fallback launch, whose one-thread-per-
+    //     row kernel moves the reference; nothing here is rescaled.
+    // At the end of an item half 1 hands its row sums to half 0, which normalises and writes O.
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(L::kRegsSoftmax));
+    const int sw = warp - 4;
+    const int qt = sw >> 3, half = (sw >> 2) & 1, wl = sw & 3;  // TMEM lanes 32 * (warp % 4) .. + 31
+    const int row = wl * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(wl * 32) << 16;
+    const uint32_t tSrow = tmem_base + lane_base + qt * kSStride;  // the row's 128 score columns
+    const uint32_t tS = tSrow + half * 64;                         // this half's; its P goes over the first 32
+    const uint32_t tO = tmem_base + lane_base + 256 + qt * 128;
+    const int sub = (R == 64) ? (wl >> 1) : 0;
+    const int my_bit = qt * kQBT + sub;
+    constexpr int kHB = (kG >= 2) ? kG / 2 : 1;   // key blocks of a half (a half block when C = 128)
+    constexpr int kBW = 64 / kHB;                 // columns per such block
+    uint64_t* const pair_bar = &ctl->pair_bar[qt * 4 + wl];
+    uint32_t nsub = 0, nod = 0, npair = 0, nitem = 0, te = 0, ent;
+
+    LOSA_TL_NEXT(ent);
+    while ((ent >> 28) == 1) {
+      const int w = (int)(ent & kTlItemMask);
+      const bool partial = (ent & kTlPartial) != 0;
+      const int part = (int)((ent >> 24) & 7u);
+      const int pbh = w / p.nPairs, pr = w % p.nPairs;
+      const int bh = pbh % (p.B * p.H);
+      const int b = bh / p.H, h = bh % p.H;
+      void* const o_base = (p.problems != nullptr) ? p.problems[pbh / (p.B * p.H)].o : p.o;
+      const int T = 2 * pr + qt;
+      const int grow = T * 128 + row;
+      float m_ref = 0.f, l = 0.f;
+      bool have_ref = false, ovf = false;
+      uint32_t pv_item = 0;
+      for (;;) {
+        uint32_t grp[kG];
+        bool more;
+        LOSA_TL_NEXT_TILE(grp, more);
+        if (!more) {
+          ent = grp[0];
+          break;
+        }
+        // hv[i]: how many columns of block i of this half the row attends to (a block is a key
+        // block, or this half's 64 columns of a 128-key block)
+        uint32_t memb = 0;
+        int hv[kHB];
+        bool mine = false, whole = true, pair_mine = false;
+#pragma unroll
+        for (int g = 0; g < kG; ++g) {
+          memb |= (grp[g] >> 16) & 0xfu;
+          pair_mine = pair_mine || ((grp[g] >> (16 + my_bit)) & 1u);
+        }
+#pragma unroll
+        for (int i = 0; i < kHB; ++i) {
+          const int g = (kG >= 2) ? half * kHB + i : 0;
+          const int jg = (int)(grp[g] & 0xffffu);
+          const int valid = ((grp[g] >> (16 + my_bit)) & 1u) ? min(kC, p.N - jg * kC) : 0;
+          hv[i] = (kG >= 2) ? valid : max(0, min(64, valid - 64 * half));
+          mine = mine || hv[i] > 0;
+          whole = whole && hv[i] == kBW;
+        }
+        if (((memb >> (qt * kQBT)) & kQMask) == 0) continue;
+        // S of this key tile is complete, and so is every earlier product into O
+        LOSA_WAIT(&ctl->s_full[qt][0], nsub & 1);
+        ptx::tc_fence_after_sync();
+        if (!have_ref && pair_mine) {
+          // the item's first tile for this row: the reference is the maximum of the row's scores
+          // over the keys it attends to, computed by both halves alike (no exchange)
+          float mx = -INFINITY;
+#pragma unroll
+          for (int c0 = 0; c0 < kW; c0 += 32) {
+            uint32_t r[32];
+            ptx::tmem_ld32(tSrow + c0, r);
+            ptx::tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const int cc = c0 + c;
+              const int jg = (int)(grp[cc / kC] & 0xffffu);
+              const int valid = ((grp[cc / kC] >> (16 + my_bit)) & 1u) ? min(kC, p.N - jg * kC) : 0;
+              if ((cc % kC) < valid) mx = fmaxf(mx, __uint_as_float(r[c]));
+            }
+          }
+          m_ref = mx * p.scale_log2;
+          have_ref = true;
+          // the other half reads the whole row too: nobody packs P over it before both are done
+          ptx::tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(pair_bar);
+          LOSA_WAIT(pair_bar, npair & 1);
+          ++npair;
+          ptx::tc_fence_after_sync();
+        }
+        uint32_t sr[64];
+        if (mine) {
+          ptx::tmem_ld32(tS, &sr[0]);
+          if (whole) ptx::tmem_wait_ld();
+          ptx::tmem_ld32(tS + 32, &sr[32]);
+          if (!whole) {
+            // keys that do not exist (>= N, in the sequence's last key block): -inf column by column
+            ptx::tmem_wait_ld();
+            bool ragged = false;
+#pragma unroll
+            for (int i = 0; i < kHB; ++i) ragged = ragged || (hv[i] > 0 && hv[i] < kBW);
+            if (ragged) {
+#pragma unroll
+              for (int c = 0; c < 64; ++c)
+                if ((c % kBW) >= hv[c / kBW]) sr[c] = 0xff800000u;
+            }
+          }
+          // key blocks the row's query block does not list get -inf as the addend of the scaling FMA
+          const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+          float2 nm2[kHB];
+#pragma unroll
+          for (int i = 0; i < kHB; ++i) {
+            const float a = (hv[i] > 0) ? -m_ref : -INFINITY;
+            nm2[i] = make_float2(a, a);
+          }
+          // The output is normalised by the sum of the weights the tensor core multiplies with V -
+          // P as rounded to bf16 - so that o is a weighted mean of V whatever the rounding does.
+          float2 racc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+          for (int c = 0; c < 64; c += 4) {
+            if (whole && c == 32) ptx::tmem_wait_ld();
+            float2 x0 = ptx::fma2(
+                make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2[c / kBW]);
+            float2 x1 = ptx::fma2(
+                make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, nm2[c / kBW]);
+            x0.x = ptx::ex2_approx(x0.x);
+            x0.y = ptx::ex2_approx(x0.y);
+            x1.x = ptx::ex2_approx(x1.x);
+            x1.y = ptx::ex2_approx(x1.y);
+            const uint32_t u0 = ptx::pack_bf16x2(x0.x, x0.y), u1 = ptx::pack_bf16x2(x1.x, x1.y);
+            sr[c >> 1] = u0;
+            sr[(c >> 1) + 1] = u1;
+            racc[0] = ptx::add2(racc[0], ptx::unpack_bf16x2(u0));
+            racc[1] = ptx::add2(racc[1], ptx::unpack_bf16x2(u1));
+          }
+          const float tsum = (racc[0].x + racc[0].y) + (racc[1].x + racc[1].y);
+          ovf = ovf || __any_sync(0xffffffffu, !(tsum <= kSplitSafeSum));
+          l += tsum;
+          ptx::tmem_st32(tS, &sr[0]);
+        } else {
+          // this half of the row lists none of the tile's keys: P = 0
+          uint32_t z[32];
+#pragma unroll
+          for (int c = 0; c < 32; ++c) z[c] = 0u;
+          ptx::tmem_st32(tS, z);
+        }
+        ptx::tmem_wait_st();
+        ++pv_item;
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&ctl->p_ready[qt]);
+        ++nsub;
+      }
+
+      // ---- end of the item: half 1 hands its row sums over, half 0 writes O / l
+      // (two sets of slots, used by alternate items: half 1 may be an item ahead of half 0's read)
+      float* const xset = ctl->xch + ((nitem & 1) * 2 + qt) * 128;
+      ++nitem;
+      if (half == 1) xset[row] = l;
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(pair_bar);
+      LOSA_WAIT(pair_bar, npair & 1);
+      ++npair;
+      if (ovf && lane == 0) {
+        // (the pair's warps may both get here, and so may the other pairs: the unit is listed once)
+        const int unit = partial ? p.split_first + (w - p.split_first) * p.split_parts + part : w;
+        if (atomicExch(&ctl->ovf_unit, unit) != unit) {
+          const int slot = atomicAdd(p.redo_count, 1);
+          if (slot < p.nUnits) p.redo_list[slot] = unit;
+        }
+      }
+      if (half == 0 && T < p.nQt) {
+        l += xset[row];
+        const bool valid = grow < p.N;
+        const float inv = (l > 0.f) ? 1.f / l : 0.f;
+        const int64_t off = (int64_t)b * p.sb + (int64_t)h * p.sh + (int64_t)grow * p.sn;
+        const int64_t pslot =
+            ((((int64_t)(w - p.split_first) * p.split_parts + part) * 2 + qt) * 128 + row);
+        if (partial) p.part_ml[pslot] = make_float2(m_ref, l);
+        if (pv_item > 0) {
+          LOSA_WAIT(&ctl->o_done[qt], nod & 1);
+          ++nod;
+          ptx::tc_fence_after_sync();
+        }
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += 32) {
+          uint32_t r[32];
+          if (pv_item > 0) {
+            ptx::tmem_ld32(tO + c0, r);
+            ptx::tmem_wait_ld();
+          } else {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) r[c] = 0u;
+          }
+          if (partial) {
+            float4* dst = reinterpret_cast<float4*>(p.part_o + pslot * D + c0);
+#pragma unroll
+            for (int c = 0; c < 32; c += 4)
+              dst[c >> 2] = make_float4(__uint_as_float(r[c]), __uint_as_float(r[c + 1]),
+                                        __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
+          } else if (valid) {
+            if (p.o_f32) {
+              float4* dst = reinterpret_cast<float4*>(static_cast<float*>(o_base) + off + c0);
+#pragma unroll
+              for (int c = 0; c < 32; c += 4)
+                dst[c >> 2] = make_float4(__uint_as_float(r[c]) * inv, __uint_as_float(r[c + 1]) * inv,
+                                          __uint_as_float(r[c + 2]) * inv,
+                                          __uint_as_float(r[c + 3]) * inv);
+            } else {
+              uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(o_base) + off + c0);
+#pragma unroll
+              for (int c = 0; c < 32; c += 8) {
+                uint4 v;
+                v.x = ptx::pack_bf16x2(__uint_as_float(r[c]) * inv, __uint_as_float(r[c + 1]) * inv);
+                v.y = ptx::pack_bf16x2(__uint_as_float(r[c + 2]) * inv, __uint_as_float(r[c + 3]) * inv);
+                v.z = ptx::pack_bf16x2(__uint_as_float(r[c + 4]) * inv, __uint_as_float(r[c + 5]) * inv);
+                v.w = ptx::pack_bf16x2(__uint_as_float(r[c + 6]) * inv, __uint_as_float(r[c + 7]) * inv);
+                dst[c >> 3] = v;
+              }
+            }
+          }
+        }
+        if (pv_item > 0) {
+          ptx::tc_fence_before_sync();
+          ptx::mbar_arrive(&ctl->o_free[qt]);
+        }
+      }
+    }
   }
 
 teardown:
@@ -1280,19 +1568,18 @@ int make_map(CUtensorMap* m, const void* base, const Geometry& g, int box_rows) 
   return LOSA_OK;
 }
 
-template <int D, int R, int C_, int MODE, int KT>
-int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Params prm, int sms,
-             cudaStream_t st) {
+// Configures (once per device) and launches one layout of the attention kernel.
+template <int D, int R, int C_, int MODE, int KT, bool SPLIT>
+int launch_kernel(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                  const Params& prm, int grid, cudaStream_t st) {
   using C = Cfg<D, R, C_, MODE, KT>;
-  using Ctl = Control<C::kNK, C::kNV>;
-  CUtensorMap mq, mk, mv;
-  int rc;
-  if ((rc = make_map(&mq, q, g, 128)) != LOSA_OK) return rc;
-  if ((rc = make_map(&mk, k, g, C::kC)) != LOSA_OK) return rc;
-  if ((rc = make_map(&mv, C::kHasV ? v : k, g, C::kC)) != LOSA_OK) return rc;
-  const size_t smem =
-      1024 + 2 * C::kQBytes + (size_t)(C::kNK + C::kNV) * C::kKVBytes + sizeof(Ctl);
-  auto kern = losa_attn_kernel<D, R, C_, MODE, KT>;
+  using L = Lay<SPLIT>;
+  using Ctl = Control<C::kNK, C::kNV, SPLIT>;
+  // (one thread per row: 1024 bytes of slack to align the tiles; two threads per row: none left,
+  // the kernel checks the alignment of its shared memory instead)
+  const size_t smem = (SPLIT ? 0 : 1024) + 2 * C::kQBytes +
+                      (size_t)(C::kNK + C::kNV) * C::kKVBytes + sizeof(Ctl);
+  auto kern = losa_attn_kernel<D, R, C_, MODE, KT, SPLIT>;
   // (function attributes belong to a device: one flag per device ordinal)
   static bool configured_on[kMaxDevices] = {};
   int dev = 0;
@@ -1302,13 +1589,27 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
     // the in-kernel register reallocation must fit the registers the CTA is launched with
     cudaFuncAttributes attr;
     LOSA_CUDA_TRY(cudaFuncGetAttributes(&attr, kern));
-    if (attr.numRegs * kThreads < 128 * kRegsUtility + 256 * kRegsSoftmax) {
+    if (attr.numRegs * L::kThreads < 128 * L::kRegsUtility + 32 * L::kSoftmaxWarps * L::kRegsSoftmax) {
       set_cuda_error(cudaErrorLaunchOutOfResources, "register budget of losa_attn_kernel");
       return LOSA_ERR_UNSUPPORTED;
     }
     LOSA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     configured = true;
   }
+  kern<<<grid, L::kThreads, smem, st>>>(mq, mk, mv, prm);
+  LOSA_CUDA_TRY(cudaGetLastError());
+  return LOSA_OK;
+}
+
+template <int D, int R, int C_, int MODE, int KT>
+int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Params prm, int sms,
+             cudaStream_t st) {
+  using C = Cfg<D, R, C_, MODE, KT>;
+  CUtensorMap mq, mk, mv;
+  int rc;
+  if ((rc = make_map(&mq, q, g, 128)) != LOSA_OK) return rc;
+  if ((rc = make_map(&mk, k, g, C::kC)) != LOSA_OK) return rc;
+  if ((rc = make_map(&mv, C::kHasV ? v : k, g, C::kC)) != LOSA_OK) return rc;
   const int ctas = min(sms, kMaxPersistentCtas);
   // The items of the last, partly filled wave of the persistent grid (all items, if there are
   // fewer than CTAs) are cut into parts of the key range, so that the wave ends after 1/parts of
@@ -1317,7 +1618,8 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
   prm.nUnits = prm.nWork;
   prm.split_first = prm.nWork;
   prm.split_parts = 1;
-  if (MODE == kDense || MODE == kSparse) {
+  constexpr bool kAttnOnly = (MODE == kDense || MODE == kSparse);
+  if (kAttnOnly) {
     const int rest = (prm.nWork < ctas) ? prm.nWork : prm.nWork % ctas;
     int parts = rest > 0 ? ctas / rest : 1;
     parts = min(min(parts, kMaxParts), prm.nKb);
@@ -1333,8 +1635,22 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
     build_tile_lists_kernel<C::kNB, C::kG><<<prm.nUnits, 32, bm_bytes, st>>>(prm);
     LOSA_CUDA_TRY(cudaGetLastError());
   }
-  kern<<<grid, kThreads, smem, st>>>(mq, mk, mv, prm);
-  LOSA_CUDA_TRY(cudaGetLastError());
+  if constexpr (kAttnOnly) {
+    // The attention-only modes run with two threads per query row and a reference that never
+    // moves; the units whose scores outgrew it (none, on ordinary inputs) are listed, and a second
+    // launch of the one-thread-per-row kernel, which returns at once when the list is empty,
+    // recomputes them with a moving reference.
+    prm.redo = 0;
+    if ((rc = launch_kernel<D, R, C_, MODE, KT, true>(mq, mk, mv, prm, grid, st)) != LOSA_OK) return rc;
+    if (!prm.stall) {
+      prm.redo = 1;
+      prm.work_counter += 2;  // its own counter (zeroed with the first)
+      if ((rc = launch_kernel<D, R, C_, MODE, KT, false>(mq, mk, mv, prm, grid, st)) != LOSA_OK) return rc;
+    }
+  } else {
+    prm.redo = 0;
+    if ((rc = launch_kernel<D, R, C_, MODE, KT, false>(mq, mk, mv, prm, grid, st)) != LOSA_OK) return rc;
+  }
   if (prm.split_parts > 1) {
     merge_parts_kernel<D><<<dim3(prm.nWork - prm.split_first, 16), 128, 0, st>>>(prm);
     LOSA_CUDA_TRY(cudaGetLastError());
@@ -1391,6 +1707,8 @@ size_t attn_workspace_bytes(AttnMode mode, const Geometry& g, int n_prob) {
     if (mode == kSparse) bytes += tl_count_bytes(g, n_prob) + tl_entries_bytes(g, n_prob);
     // batched launch: the table of the problems' tensor maps and pointers
     if (n_prob > 1) bytes += (size_t)n_prob * sizeof(ProblemEntry);
+    // the work units handed to the fallback launch
+    bytes += tl_count_bytes(g, n_prob);
     return bytes;
   }
   // counter, per-CTA row statistics, per-CTA table of one entry per row and key tile
@@ -1458,6 +1776,11 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
       k = layers[0].k;
       v = layers[0].v;
     }
+    // counter block: [0] work counter, [1] length of the fallback list, [2] the fallback launch's counter
+    prm.redo_count = prm.work_counter + 1;
+    prm.redo_list = reinterpret_cast<int*>(
+        tl + (mode == kSparse ? tl_count_bytes(g, n_prob) + tl_entries_bytes(g, n_prob) : 0) +
+        (n_prob > 1 ? (size_t)n_prob * sizeof(ProblemEntry) : 0));
   }
   prm.scale_log2 = g.scale * kLog2e;
   int rc = LOSA_OK;
@@ -1469,7 +1792,7 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
   const uint32_t stall_polls = g_stall_polls.exchange(0u);
   prm.stall = stall_polls > 0u ? 1 : 0;
   prm.wait_polls = stall_polls > 0u ? stall_polls : ptx::kWaitPolls;
-  LOSA_CUDA_TRY(cudaMemsetAsync(prm.work_counter, 0, sizeof(int), st));
+  LOSA_CUDA_TRY(cudaMemsetAsync(prm.work_counter, 0, 4 * sizeof(int), st));
   switch (mode) {
     case kDense: return dispatch<kDense>(g, q, k, v, prm, sms, st);
     case kSparse: return dispatch<kSparse>(g, q, k, v, prm, sms, st);
