@@ -456,7 +456,10 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // softmax warps as soon as it is read.
     {
       const int qt = warp - kIssuerWarp;
-      const bool leader = (lane == 0);
+      // The leader comes from elect.sync rather than from a lane test: the compiler then knows that
+      // a single thread runs the issue code and keeps the MMA operands in uniform registers, which
+      // halves the cost of issuing an MMA (measured: 27 instead of 55-65 cycles per instruction).
+      const bool leader = ptx::elect_one();
       uint32_t nq = 0, nt = 0, nsub = 0, nof = 0, te = 0, ent;
       constexpr uint32_t kDescHi = ptx::smem_desc_hi_sw128(1024);
       const uint32_t k_lo = ptx::smem_desc_lo(ptx::smem_u32(sK), 16);
@@ -1293,7 +1296,8 @@ teardown:
   if (ctl->abort_flag) {
     // Abort path: give MMAs and bulk copies still in flight a bounded time to land before
     // shared memory and TMEM are released.
-    if ((warp == kIssuerWarp || warp == kIssuerWarp + 1) && lane == 0) {
+    // (the same thread that issued the MMAs: the election is deterministic for a full warp)
+    if ((warp == kIssuerWarp || warp == kIssuerWarp + 1) && ptx::elect_one()) {
       ptx::mma_commit(&ctl->drain);
       for (uint32_t it = 0; it < (1u << 16); ++it) {
         if (ptx::mbar_try_wait(&ctl->drain, 0)) break;
