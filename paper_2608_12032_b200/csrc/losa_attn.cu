@@ -95,7 +95,7 @@ constexpr float kSafeRowSum = 1.099511627776e12f;  // 2^40: a tile's row sum bey
 // two threads per row: a tile's half-row sum beyond 2^60 (or NaN) sends the work unit to the fallback
 constexpr float kSplitSafeSum = 1.152921504606846976e18f;
 
-template <int D, int R, int C_, int MODE, int KT>
+template <int D, int R, int C_, int MODE, int KT, bool ROT = false>
 struct Cfg {
   static constexpr int kC = C_;                       // keys per key block
   static constexpr int kT = KT;                       // keys per K/V tile: one S = Q K^T per tile
@@ -118,9 +118,11 @@ struct Cfg {
   static constexpr int kRingBudget = (kHasV ? 160 : 128) * 1024;  // K + V rings
   // a V tile stays in use about one tile longer than a K tile (its product is issued after the
   // tile's softmax), so V gets the deeper ring
-  static constexpr int kNV = kHasV ? ((kKVBytes >= 32768) ? 3 : 4) : 0;
+  // (rotating score buffers, head dimension 64: O += P V trails S = Q K^T by up to three steps, so
+  // a V tile is held that much longer while a K tile goes back at once: 7 V and 4 K stages of 16 KB)
+  static constexpr int kNV = ROT ? 7 : kHasV ? ((kKVBytes >= 32768) ? 3 : 4) : 0;
   static constexpr int kNK0 = (kRingBudget - kNV * kKVBytes) / kKVBytes;
-  static constexpr int kNK = kNK0 > 6 ? 6 : kNK0;
+  static constexpr int kNK = ROT ? 4 : kNK0 > 6 ? 6 : kNK0;
   static constexpr uint32_t kIdescQK = ptx::idesc_bf16_f32(128, kW, false, false);
   static constexpr uint32_t kIdescPV = ptx::idesc_bf16_f32(128, D, false, true);
 };
@@ -173,7 +175,7 @@ struct Params {
   int stall;            // diagnostic launch: the scheduler publishes nothing, so that every wait runs out
 };
 
-template <int NK, int NV, bool SPLIT>
+template <int NK, int NV, bool SPLIT, bool ROT>
 struct Control {
   uint64_t q_full[2], q_empty[2];
   uint64_t k_full[NK], k_empty[NK];
@@ -194,6 +196,12 @@ struct Control {
   uint64_t pair_bar[SPLIT ? 8 : 1];
   float xch[SPLIT ? 2 * 2 * 128 : 1];
   int ovf_unit;
+  // head dimension 64, two threads per row: three score buffers used in turn by both query tiles.
+  // One barrier per (query tile, buffer): a barrier's phases then follow one query tile's own
+  // sequence of tiles, so that its warps are never more than one phase away from it (they may be
+  // whole work units ahead of, or behind, the other query tile's warps).
+  uint64_t rot_s_full[ROT ? 6 : 1], rot_p_ready[ROT ? 6 : 1];
+  uint64_t pv_done[ROT ? 3 : 1];  // per buffer: the product that read its P has run
 };
 
 #define LOSA_WAIT_RELAXED(bar, parity)                                   \
@@ -277,10 +285,18 @@ template <int D, int R, int C_, int MODE, int KT, bool SPLIT>
 __global__ void __launch_bounds__(Lay<SPLIT>::kThreads, 1)
 losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, const Params p) {
-  using C = Cfg<D, R, C_, MODE, KT>;
+  using C = Cfg<D, R, C_, MODE, KT, SPLIT && D == 64>;
   using L = Lay<SPLIT>;
-  using Ctl = Control<C::kNK, C::kNV, SPLIT>;
+  using Ctl = Control<C::kNK, C::kNV, SPLIT, SPLIT && D == 64>;
   static_assert(!SPLIT || (C::kHasV && !C::kWantMass), "two threads per row: attention-only modes");
+  // Head dimension 64 leaves 128 tensor-memory columns unused (O takes 64 per query tile), enough
+  // for a third score buffer.  The two query tiles then take the three buffers in turn, in the
+  // order in which their S = Q K^T are issued, so that the S of a query tile's next key tile is
+  // computed while its current one is still being exponentiated: the softmax warps never wait for
+  // the tensor core.  One issuer warp issues every S = Q K^T of the CTA in that fixed order, the
+  // other every O += P V; a buffer is written again only after the product that read its P has
+  // completed (a barrier between the two issuers).
+  constexpr bool kRot = SPLIT && D == 64;
   constexpr int kC = C::kC, kG = C::kG, kQBT = C::kQBT, kNB = C::kNB, kW = C::kW, kNS = C::kNS;
   constexpr uint32_t kSStride = C::kSStride, kNVs = C::kNV > 0 ? C::kNV : 1;
   constexpr uint32_t kQMask = (1u << kQBT) - 1u;
@@ -336,6 +352,13 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     if (SPLIT) {
       for (int i = 0; i < 8; ++i) ptx::mbar_init(&ctl->pair_bar[i], 2);
       ctl->ovf_unit = -1;
+    }
+    if (kRot) {
+      for (int i = 0; i < 3; ++i) ptx::mbar_init(&ctl->pv_done[i], 1);
+      for (int i = 0; i < 6; ++i) {
+        ptx::mbar_init(&ctl->rot_s_full[i], 1);
+        ptx::mbar_init(&ctl->rot_p_ready[i], L::kSoftmaxWarps / 2);
+      }
     }
     ptx::mbar_init(&ctl->drain, 2);  // the MMA issuers arrive on the abort path
     ctl->mma_lock = 0;
@@ -438,6 +461,135 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                                &ctl->v_full[vs], s * 64, r0, h, b);
             }
             ++nv;
+          }
+        }
+      }
+    }
+  } else if (kRot && warp == kIssuerWarp) {
+    // ------------------------------------------------------------------ rotating score buffers: the S = Q K^T issuer
+    // For every K/V tile of the list, for each query tile that lists it (query tile 0 first): the
+    // next score, number k, goes into buffer k % 3.  That buffer still holds the P of score
+    // k - 3 until its O += P V has run, which the other issuer warp signals (pv_done).
+    {
+      const bool leader = ptx::elect_one();
+      constexpr uint32_t kDescHi = ptx::smem_desc_hi_sw128(1024);
+      const uint32_t k_lo = ptx::smem_desc_lo(ptx::smem_u32(sK), 16);
+      const uint32_t q_lo = ptx::smem_desc_lo(ptx::smem_u32(sQ), 16);
+      uint32_t nq[2] = {0, 0}, nt = 0, te = 0, ent, kq = 0;
+      LOSA_TL_NEXT(ent);
+      while ((ent >> 28) == 1) {
+        bool q_ready[2] = {false, false};
+        const int pr_ = (int)(ent & kTlItemMask) % p.nPairs;
+        for (;;) {
+          uint32_t grp[kG];
+          bool more;
+          LOSA_TL_NEXT_TILE(grp, more);
+          if (!more) {
+            ent = grp[0];
+            break;
+          }
+          uint32_t memb = 0;
+#pragma unroll
+          for (int g = 0; g < kG; ++g) memb |= (grp[g] >> 16) & 0xfu;
+          const uint32_t ks = nt % C::kNK, kph = (nt / C::kNK) & 1;
+          LOSA_WAIT(&ctl->k_full[ks], kph);
+#pragma unroll
+          for (int qt = 0; qt < 2; ++qt) {
+            if (((memb >> (qt * kQBT)) & kQMask) != 0) {
+              if (!q_ready[qt]) {
+                LOSA_WAIT(&ctl->q_full[qt], nq[qt] & 1);
+                ++nq[qt];
+                q_ready[qt] = true;
+              }
+              const uint32_t b = kq % 3u;
+              if (kq >= 3u) LOSA_WAIT(&ctl->pv_done[b], (kq / 3u - 1u) & 1);
+              ptx::tc_fence_after_sync();
+              if (leader) {
+                const uint32_t qd0 = q_lo + qt * (C::kQBytes >> 4), kd0 = k_lo + ks * (C::kKVBytes >> 4);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk)
+                  ptx::mma_ss_lo(tmem_base + b * 128, qd0 + (((kk >> 2) * C::kQSlab + (kk & 3) * 32) >> 4),
+                                 kd0 + (((kk >> 2) * C::kKVSlab + (kk & 3) * 32) >> 4), kDescHi,
+                                 C::kIdescQK, kk > 0 ? 1u : 0u);
+                ptx::mma_commit(&ctl->rot_s_full[qt * 3 + b]);
+                ptx::mma_commit(&ctl->k_empty[ks]);
+              }
+              ++kq;
+            } else {
+              if (leader) ptx::mbar_arrive(&ctl->k_empty[ks]);
+            }
+          }
+          ++nt;
+        }
+#pragma unroll
+        for (int qt = 0; qt < 2; ++qt) {
+          if (q_ready[qt]) {
+            if (leader) ptx::mma_commit(&ctl->q_empty[qt]);
+          } else if (2 * pr_ + qt < p.nQt) {
+            // no key tile of this unit was listed by the query tile: its buffer goes back unused
+            LOSA_WAIT(&ctl->q_full[qt], nq[qt] & 1);
+            ++nq[qt];
+            if (leader) ptx::mbar_arrive(&ctl->q_empty[qt]);
+          }
+        }
+      }
+    }
+  } else if (kRot && warp == kIssuerWarp + 1) {
+    // ------------------------------------------------------------------ rotating score buffers: the O += P V issuer
+    // Walks the same list in the same order; product k reads P from buffer k % 3 once the softmax
+    // warps of its query tile have packed it.
+    {
+      const bool leader = ptx::elect_one();
+      constexpr uint32_t kDescHi = ptx::smem_desc_hi_sw128(1024);
+      const uint32_t v_lo = ptx::smem_desc_lo(ptx::smem_u32(sV), C::kKVSlab);
+      uint32_t nof[2] = {0, 0}, uses[6] = {0, 0, 0, 0, 0, 0}, nt = 0, te = 0, ent, kp = 0;
+      LOSA_TL_NEXT(ent);
+      while ((ent >> 28) == 1) {
+        uint32_t pv_item[2] = {0, 0};
+        for (;;) {
+          uint32_t grp[kG];
+          bool more;
+          LOSA_TL_NEXT_TILE(grp, more);
+          if (!more) {
+            ent = grp[0];
+            break;
+          }
+          uint32_t memb = 0;
+#pragma unroll
+          for (int g = 0; g < kG; ++g) memb |= (grp[g] >> 16) & 0xfu;
+          const uint32_t vs = nt % kNVs, vph = (nt / kNVs) & 1;
+          LOSA_WAIT(&ctl->v_full[vs], vph);
+#pragma unroll
+          for (int qt = 0; qt < 2; ++qt) {
+            if (((memb >> (qt * kQBT)) & kQMask) != 0) {
+              const uint32_t b = kp % 3u;
+              if (pv_item[qt] == 0 && nof[qt] > 0) LOSA_WAIT(&ctl->o_free[qt], (nof[qt] - 1) & 1);
+              LOSA_WAIT(&ctl->rot_p_ready[qt * 3 + b], uses[qt * 3 + b] & 1);
+              ++uses[qt * 3 + b];
+              ptx::tc_fence_after_sync();
+              if (leader) {
+                const uint32_t tP = tmem_base + b * 128, tO = tmem_base + 384 + qt * 64;
+                const uint32_t vd0 = v_lo + vs * (C::kKVBytes >> 4);
+#pragma unroll
+                for (int kk = 0; kk < kW / 16; ++kk)
+                  ptx::mma_ts_lo(tO, tP + (kk & 3) * 8 + (kk >> 2) * 64, vd0 + kk * (2048 >> 4), kDescHi,
+                                 C::kIdescPV, (kk > 0 || pv_item[qt] > 0) ? 1u : 0u);
+                ptx::mma_commit(&ctl->pv_done[b]);
+                ptx::mma_commit(&ctl->v_empty[vs]);
+              }
+              ++pv_item[qt];
+              ++kp;
+            } else {
+              if (leader) ptx::mbar_arrive(&ctl->v_empty[vs]);
+            }
+          }
+          ++nt;
+        }
+#pragma unroll
+        for (int qt = 0; qt < 2; ++qt) {
+          if (pv_item[qt] > 0) {
+            if (leader) ptx::mma_commit(&ctl->o_done[qt]);  // every product of the item is done
+            ++nof[qt];
           }
         }
       }
@@ -1070,9 +1222,13 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int qt = sw >> 3, half = (sw >> 2) & 1, wl = sw & 3;  // TMEM lanes 32 * (warp % 4) .. + 31
     const int row = wl * 32 + lane;
     const uint32_t lane_base = (uint32_t)(wl * 32) << 16;
-    const uint32_t tSrow = tmem_base + lane_base + qt * kSStride;  // the row's 128 score columns
-    const uint32_t tS = tSrow + half * 64;                         // this half's; its P goes over the first 32
-    const uint32_t tO = tmem_base + lane_base + 256 + qt * 128;
+    // the row's 128 score columns, and this half's 64 of them (its P goes over their first 32);
+    // with rotating buffers (head dimension 64) they change from tile to tile
+    uint32_t tSrow = tmem_base + lane_base + qt * kSStride;
+    uint32_t tS = tSrow + half * 64;
+    const uint32_t tO = tmem_base + lane_base + (kRot ? 384 + qt * 64 : 256 + qt * 128);
+    uint32_t kq = 0;  // rotating buffers: scores issued so far, counted as the issuer counts them
+    uint32_t uses[3] = {0, 0, 0};  // ... and how many of them, per buffer, were this query tile's
     const int sub = (R == 64) ? (wl >> 1) : 0;
     const int my_bit = qt * kQBT + sub;
     constexpr int kHB = (kG >= 2) ? kG / 2 : 1;   // key blocks of a half (a half block when C = 128)
@@ -1121,9 +1277,27 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           mine = mine || hv[i] > 0;
           whole = whole && hv[i] == kBW;
         }
-        if (((memb >> (qt * kQBT)) & kQMask) == 0) continue;
-        // S of this key tile is complete, and so is every earlier product into O
-        LOSA_WAIT(&ctl->s_full[qt][0], nsub & 1);
+        uint32_t rot_b = 0;
+        if (kRot) {
+          // the buffer follows from the tile's place in the issue order: per K/V tile, query tile 0
+          // first, then query tile 1, each only if it lists the tile
+          const bool m0 = (memb & kQMask) != 0, m1 = ((memb >> kQBT) & kQMask) != 0;
+          const uint32_t kmine = kq + ((qt == 1 && m0) ? 1u : 0u);
+          kq += (m0 ? 1u : 0u) + (m1 ? 1u : 0u);
+          if (!(qt == 0 ? m0 : m1)) continue;
+          rot_b = kmine % 3u;
+          tSrow = tmem_base + lane_base + rot_b * 128;
+          tS = tSrow + half * 64;
+          const uint32_t par = (rot_b == 0 ? uses[0] : rot_b == 1 ? uses[1] : uses[2]) & 1;
+          uses[0] += (rot_b == 0);
+          uses[1] += (rot_b == 1);
+          uses[2] += (rot_b == 2);
+          LOSA_WAIT(&ctl->rot_s_full[qt * 3 + rot_b], par);
+        } else {
+          if (((memb >> (qt * kQBT)) & kQMask) == 0) continue;
+          // S of this key tile is complete, and so is every earlier product into O
+          LOSA_WAIT(&ctl->s_full[qt][0], nsub & 1);
+        }
         ptx::tc_fence_after_sync();
         if (!have_ref && pair_mine) {
           // the item's first tile for this row: the reference is the maximum of the row's scores
@@ -1212,7 +1386,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         ++pv_item;
         ptx::tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&ctl->p_ready[qt]);
+        if (lane == 0) ptx::mbar_arrive(kRot ? &ctl->rot_p_ready[qt * 3 + rot_b] : &ctl->p_ready[qt]);
         ++nsub;
       }
 
@@ -1576,13 +1750,15 @@ int make_map(CUtensorMap* m, const void* base, const Geometry& g, int box_rows) 
 template <int D, int R, int C_, int MODE, int KT, bool SPLIT>
 int launch_kernel(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                   const Params& prm, int grid, cudaStream_t st) {
-  using C = Cfg<D, R, C_, MODE, KT>;
+  using C = Cfg<D, R, C_, MODE, KT, SPLIT && D == 64>;
   using L = Lay<SPLIT>;
-  using Ctl = Control<C::kNK, C::kNV, SPLIT>;
+  using Ctl = Control<C::kNK, C::kNV, SPLIT, SPLIT && D == 64>;
   // (one thread per row: 1024 bytes of slack to align the tiles; two threads per row: none left,
   // the kernel checks the alignment of its shared memory instead)
   const size_t smem = (SPLIT ? 0 : 1024) + 2 * C::kQBytes +
                       (size_t)(C::kNK + C::kNV) * C::kKVBytes + sizeof(Ctl);
+  static_assert((SPLIT ? 0 : 1024) + 2 * C::kQBytes + (C::kNK + C::kNV) * C::kKVBytes + sizeof(Ctl) <= 227 * 1024,
+                "shared memory of one CTA");
   auto kern = losa_attn_kernel<D, R, C_, MODE, KT, SPLIT>;
   // (function attributes belong to a device: one flag per device ordinal)
   static bool configured_on[kMaxDevices] = {};
