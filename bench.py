@@ -15,11 +15,14 @@ the retained blocks only.  Everything is timed with CUDA events on the launching
     python bench.py --impl reference ...      # the fp64 CPU oracle on a bounded sample
 
 Under torchrun every rank runs the same layer shape on its own seeds (weak scaling; the path has
-no exchange step, so there is no data-path collective) and rank 0 prints one JSON line.
+no exchange step, so there is no data-path collective) and rank 0 prints one JSON line.  With
+`--shard heads` the ranks split the heads of ONE layer instead (strong scaling, still no collective:
+every head is independent and a CSR row belongs to one head).
 """
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -39,20 +42,42 @@ from paper_2608_12032_b200 import inputs  # noqa: E402
 METRIC = "block_sparse_attn_effective_tflops"
 UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one sparse-forward launch, from the ncu capture
-# summarised in profiles/losa_attn_kernel_wan_ncu.md (not re-measured by this script)
+# dram__bytes_read.sum + dram__bytes_write.sum of one sparse-forward launch, from an ncu capture of
+# the same kernel on the same workload (a profiler run: not re-measured by this script, which never
+# runs under a profiler); None where no capture was taken
 NCU_DRAM_BYTES_PER_LAUNCH = {"wan": 0.305036e9 + 0.086246e9}
+NCU_TRAFFIC_SOURCE = "ncu capture of the sparse forward at the Wan2.1 shape (dram__bytes_read.sum + dram__bytes_write.sum)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
 def merge_kernel_runs(wl) -> bool:
-    """Whether the attention-only calls launch their second (merge) kernel for this shape: the host
-    rule of the library, restated (work items = pairs of 128-row query tiles per head)."""
+    """Whether the attention-only calls launch their merge kernel for this shape: the host rule of
+    the library, restated (work items = pairs of 128-row query tiles per head)."""
     ctas = min(torch.cuda.get_device_properties(0).multi_processor_count, 160)
     n_work = wl.B * wl.H * ((-(-wl.N // 128) + 1) // 2)
     rest = n_work if n_work < ctas else n_work % ctas
     parts = min(ctas // rest, 8, -(-wl.N // wl.C)) if rest else 1
     return parts >= 2
+
+
+def launches_per_step(wl, draws: int) -> int:
+    """Kernels of the library launched by one step: mass 1; select 3; every sparse call its tile-list
+    pre-pass, the attention kernel and the fallback kernel behind it (which returns at once when no
+    row outgrew its reference), plus the merge kernel when the last wave is cut into parts; the
+    dense call the same without the pre-pass; the fused construction step 1."""
+    merge = int(merge_kernel_runs(wl))
+    return 1 + 3 + draws * (3 + merge) + (2 + merge) + 1
+
+
+def cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
 
 
 def parse_args():
@@ -65,6 +90,11 @@ def parse_args():
     ap.add_argument("--draws", type=int, default=10, help="reuse draws per step")
     ap.add_argument("--tau", type=float, default=None)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-baseline sample")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
+                    help="N > 1: every rank its own layer (weak scaling), or the heads of one layer split "
+                         "across the ranks (strong scaling); no collective inside the path either way")
+    ap.add_argument("--batched-layers", type=int, default=0,
+                    help="also time losa_sparse_attn_batched over this many layers against the single calls")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -163,14 +193,24 @@ def max_over_ranks(values, dist, device):
     return [float(x) for x in t.cpu()]
 
 
+def sum_over_ranks(value: float, dist, device) -> float:
+    """Sum of one float over all ranks (identity without a process group)."""
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.cpu()[0])
+
+
 def aggregate_tflops(flops_per_call: float, calls: int, slowest_rank_ms: float, world: int) -> float:
     """Whole-job throughput: every rank does `calls` launches of `flops_per_call`; the job takes as
     long as its slowest rank (weak scaling, no exchange between ranks)."""
     return world * flops_per_call * calls / (slowest_rank_ms * 1e-3) / 1e12
 
 
-def cpu_baseline(wl, q, k, v, offsets, kv_idx, seconds: float):
-    """The oracle's sparse attention (Eq. 4), as it stands, on a bounded sample of query blocks."""
+def cpu_baseline(wl, q, k, v, offsets, kv_idx, seconds: float, gpu_mass=None, tau=None):
+    """The oracle, as it stands, on a bounded sample of query blocks: its sparse attention (Eq. 4)
+    is the baseline value; its dense attention, block mass and selection are timed beside it on a
+    few blocks, and the GPU's pattern is checked against the oracle's rule on the GPU's own masses."""
     from oracle import losa_oracle as orc
 
     qn, kn, vn = (t.float().numpy() for t in (q, k, v))
@@ -193,16 +233,57 @@ def cpu_baseline(wl, q, k, v, offsets, kv_idx, seconds: float):
         if time.perf_counter() - t0 >= seconds:
             break
     dt = time.perf_counter() - t0
-    return {
+    out = {
         "value": flops / dt / 1e12,
         "unit": UNIT,
         "cores": orc.threads(),
+        "cpu": cpu_model(),
         "kind": "oracle",
         "sample": f"fp64 oracle sparse attention on {done} of {rows} query blocks "
                   f"(random sample, seed 0) of the {wl.name} workload in {dt:.1f} s",
         "seconds": dt,
         "blocks": done,
     }
+    # the other steps, each on a handful of blocks: seconds per query block and per full layer
+    few = np.sort(order[: max(2, min(8, orc.threads() // 4))]).astype(np.int32)
+    per_block = {"sparse_attn": dt / max(done, 1)}
+    t0 = time.perf_counter()
+    mass_few = orc.block_mass(qn, kn, wl.R, wl.C, row_ids=few)
+    per_block["block_mass"] = (time.perf_counter() - t0) / len(few)
+    counts = np.ones(rows, dtype=np.int64)
+    counts[few] = wl.nKb
+    doff = np.zeros(rows + 1, dtype=np.int64)
+    np.cumsum(counts, out=doff[1:])
+    didx = np.zeros(doff[-1], dtype=np.int32)
+    for r in few:
+        didx[doff[r]:doff[r + 1]] = np.arange(wl.nKb)
+    t0 = time.perf_counter()
+    orc.sparse_attn(qn, kn, vn, wl.R, wl.C, doff.astype(np.int32), didx, row_ids=few)
+    per_block["dense_attn"] = (time.perf_counter() - t0) / len(few)
+    out["oracle_seconds_per_query_block"] = per_block
+    out["oracle_seconds_per_layer_extrapolated"] = {k_: v_ * rows for k_, v_ in per_block.items()}
+    if gpu_mass is not None:
+        # selection on every row of the GPU's own masses: oracle seconds, CSR equality, near-tau rows
+        t0 = time.perf_counter()
+        sel = orc.select(gpu_mass.astype(np.float64), tau)
+        out["oracle_seconds_per_layer_extrapolated"]["select"] = time.perf_counter() - t0
+        dist = sel.boundary_distance()
+        ref_off = sel.offsets
+        same = bool(np.array_equal(ref_off, offsets)) and bool(np.array_equal(sel.kv_idx, kv_idx[: offsets[-1]]))
+        mism = 0
+        if not same:
+            for r in range(rows):
+                a = kv_idx[offsets[r]:offsets[r + 1]]
+                b = sel.kv_idx[ref_off[r]:ref_off[r + 1]]
+                if a.shape != b.shape or not np.array_equal(a, b):
+                    mism += 1
+        out["select_check"] = {
+            "rows": int(rows), "csr_equals_oracle_rule_on_gpu_masses": same, "rows_that_differ": int(mism),
+            "rows_within_1e-6_of_tau": int((dist < 1e-6).sum()),
+            "min_distance_to_tau": float(dist.min()),
+        }
+        del mass_few
+    return out
 
 
 def run_reference(args, wl, rank, world):
@@ -288,7 +369,9 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     tau = wl.tau if args.tau is None else args.tau
-    base_seed = 1000 * rank  # rank r draws its own layer
+    shard_heads = args.shard == "heads" and world > 1
+    # replicas: rank r draws its own layer; heads: every rank draws the same layer and keeps its heads
+    base_seed = 0 if shard_heads else 1000 * rank
     peaks = load_peaks()
 
     # ---- inputs: step-0 tensors and the reuse draws, resident in HBM before timing starts
@@ -296,6 +379,16 @@ def main():
     q0, k0, v0 = (t.bfloat16() for t in base)
     host_draws = [inputs.make_reuse_draw(wl, base_seed + t, base=base) for t in range(1, args.draws + 1)]
     del base
+    full_heads = wl.H
+    if shard_heads:
+        # heads [h0, h1) of the layer: every (batch, head) is independent in all four calls and a CSR
+        # row belongs to one head, so the ranks exchange nothing inside the path
+        from paper_2608_12032_b200 import sharding
+
+        h0, h1 = sharding.head_range(wl.H, rank, world)
+        q0, k0, v0 = (sharding.shard_heads(t, rank, world).contiguous() for t in (q0, k0, v0))
+        host_draws = [tuple(sharding.shard_heads(t, rank, world).contiguous() for t in d) for d in host_draws]
+        wl = dataclasses.replace(wl, H=h1 - h0)
     q0d, k0d = q0.to(dev), k0.to(dev)
     draws = [tuple(t.to(dev) for t in d) for d in host_draws]
 
@@ -372,7 +465,53 @@ def main():
 
     total_ms_max, sparse_total_ms_max = max_over_ranks([total_ms, sparse_total_ms], dist, dev)
     n_sparse_calls = args.steps * args.draws
-    value = aggregate_tflops(flops_sparse, n_sparse_calls, sparse_total_ms_max, world)
+    if shard_heads:
+        # strong scaling: the job is ONE layer; its flops are the sum of the ranks' shares
+        flops_job = sum_over_ranks(flops_sparse, dist, dev)
+        value = flops_job * n_sparse_calls / (sparse_total_ms_max * 1e-3) / 1e12
+    else:
+        value = aggregate_tflops(flops_sparse, n_sparse_calls, sparse_total_ms_max, world)
+
+    # ---- Recall (Eq. 2) of the frozen pattern: at the construction step and on every reuse draw
+    # (outside the timed region: it needs the block masses of every draw)
+    def recall_of(qd_, kd_):
+        m = losa.losa_block_mass(qd_, kd_, wl.R, wl.C, ws=ws_mass, mass=mass_fused)
+        ret, tot = losa.losa_row_recall(m, offsets, kv_idx)
+        return float(ret.sum() / tot.sum()), float((ret / tot).min())
+
+    recall0 = recall_of(q0d, k0d)
+    recall_draws = [recall_of(d[0], d[1]) for d in draws]
+    losa.check_async("recall")
+    gpu_mass_h = mass.cpu().numpy().reshape(rows, nKb)
+
+    # ---- several layers in one launch against the same layers one call each (optional)
+    batched = None
+    if args.batched_layers > 1:
+        L = args.batched_layers
+        layers = [draws[i % len(draws)] + (offsets, kv_idx) for i in range(L)]
+        outs = [torch.empty_like(draws[0][0]) for _ in range(L)]
+        ws_b = torch.empty(losa.losa_workspace_bytes_batched(2, prob, L), dtype=torch.uint8, device=dev)
+
+        def timed(fn, reps=20):
+            for _ in range(3):
+                fn()
+            a, b = ev(), ev()
+            a.record()
+            for _ in range(reps):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+
+        def singles():
+            for (q, k, v, o_, i_), o in zip(layers, outs):
+                losa.losa_sparse_attn(q, k, v, o_, i_, wl.R, wl.C, out=o, ws=ws_attn)
+
+        ms_single = timed(singles)
+        ms_batched = timed(lambda: losa.losa_sparse_attn_batched(layers, wl.R, wl.C, outs=outs, ws=ws_b))
+        losa.check_async("batched")
+        batched = {"layers": L, "ms_single_calls": ms_single, "ms_one_launch": ms_batched,
+                   "speedup": ms_single / ms_batched}
 
     # ---- end to end through the public API with host buffers (pinned), copies inside the timing
     e2e = None
@@ -433,7 +572,8 @@ def main():
         (e2e_ms,) = max_over_ranks([a.elapsed_time(b)], dist, dev)
         nbytes = q0.numel() * 2
         e2e = {
-            "value": aggregate_tflops(flops_sparse, args.draws * n_e2e, e2e_ms, world),
+            "value": (sum_over_ranks(flops_sparse, dist, dev) * args.draws * n_e2e / (e2e_ms * 1e-3) / 1e12
+                      if shard_heads else aggregate_tflops(flops_sparse, args.draws * n_e2e, e2e_ms, world)),
             "unit": UNIT,
             "h2d_bytes_per_step": (2 + 3 * args.draws) * nbytes,
             "d2h_bytes_per_step": args.draws * nbytes,
@@ -453,18 +593,23 @@ def main():
 
     sparse_avg_ms = sparse_total_ms / n_sparse_calls
     achieved = flops_sparse / (sparse_avg_ms * 1e-3) / 1e12
-    peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+    burst = float(peaks["bf16_tflops"])
+    sustained = float(peaks.get("bf16_tflops_sustained", burst))
     dense_flops = wl.dense_flop()
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": total_ms_max / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "scaling": "strong" if shard_heads else "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
         "config": {
-            "workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "D": wl.D, "R": wl.R, "C": wl.C,
+            "workload": wl.name, "B": wl.B, "H": full_heads, "N": wl.N, "D": wl.D, "R": wl.R, "C": wl.C,
             "tau": tau, "draws": args.draws, "coverage": coverage, "nnz": int(off_h[-1]),
             "step": "block_mass + select + draws x sparse_attn + 1 dense attn + 1 fused attn_mass",
             "l2": "inputs larger than L2: each sparse call reads a different 300 MB draw",
             "pe_base": wl.pe_base, "pe_scale": wl.pe_scale,
+            "multi_gpu": ("heads of one layer split across the ranks (rank 0 reports its own share "
+                          f"of {wl.H} heads below)" if shard_heads else
+                          "every rank its own layer" if world > 1 else "one GPU"),
         },
         "ms_per_layer": {
             "sparse_attn": sparse_avg_ms, "sparse_attn_min": min(sparse_ms),
@@ -475,28 +620,34 @@ def main():
         "sparse_vs_dense_speedup": statistics.mean(dense_ms) / sparse_avg_ms,
         "dense_tflops": dense_flops / (statistics.mean(dense_ms) * 1e-3) / 1e12,
         "block_mass_tflops": 0.5 * dense_flops / (statistics.mean(mass_ms) * 1e-3) / 1e12,
+        "select_gbs": (4.0 * rows * nKb + 4.0 * (int(off_h[-1]) + rows + 1)) / (statistics.mean(sel_ms) * 1e-3) / 1e9,
+        "recall": {
+            "construction_step": recall0[0], "construction_step_min_row": recall0[1],
+            "reuse_draws": [r[0] for r in recall_draws], "reuse_draws_min_row": [r[1] for r in recall_draws],
+            "note": "Eq. 2 on the GPU's own block masses of each draw, frozen pattern from step 0",
+        },
         "roofline": {
             "kernel": "losa_attn_kernel<sparse>", "bound": "tensor", "achieved": achieved,
-            "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-            "peak_source": f"{peaks['_source']} bf16_tflops_sustained (kernel timed inside a long step)",
-            "frac_of_burst": achieved / float(peaks["bf16_tflops"]),
+            "peak": burst, "unit": "TFLOP/s", "frac": achieved / burst,
+            "peak_source": f"{peaks['_source']} bf16_tflops (cuBLAS burst)",
+            "frac_of_sustained": achieved / sustained,
             "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS,
             "flops_per_launch": flops_sparse,
             "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(wl.name),
-            "traffic_unit": "bytes per launch (DRAM read + write, ncu)",
+            "traffic_unit": "bytes per launch (DRAM read + write)",
+            "traffic_source": NCU_TRAFFIC_SOURCE if wl.name in NCU_DRAM_BYTES_PER_LAUNCH else None,
             "algorithmic_bytes_per_launch": 4 * q0.numel() * 2,
         },
         "clocks": clocks.summary(),
-        # per step: mass 1, select 3, `draws` sparse calls of 2 kernels (tile-list pre-pass + attention),
-        # dense 1, fused 1; each attention-only call adds its merge kernel when the last wave of work
-        # items is cut into parts
-        "gpu_launches": args.steps * (1 + 3 + args.draws * (2 + int(merge_kernel_runs(wl)))
-                                      + 1 + int(merge_kernel_runs(wl)) + 1),
+        "gpu_launches": args.steps * launches_per_step(wl, args.draws),
     }
+    if batched is not None:
+        line["batched"] = batched
     if e2e is not None:
         line["e2e"] = e2e
     if not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(wl, *host_draws[0], off_h, idx_h, args.cpu_seconds)
+        line["cpu_baseline"] = cpu_baseline(wl, *host_draws[0], off_h, idx_h, args.cpu_seconds,
+                                            gpu_mass=gpu_mass_h, tau=tau)
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

@@ -28,7 +28,9 @@ def _worker(rank, world, port, out):
     # rank r took (10 + 5 r) ms in total and (4 + 2 r) ms in its sparse launches
     total, sparse = bench.max_over_ranks([10.0 + 5 * rank, 4.0 + 2 * rank], dist, torch.device("cpu"))
     value = bench.aggregate_tflops(1e12, 3, sparse, world)
-    out[rank] = (total, sparse, value)
+    # heads of one layer split across the ranks: the job's flops are the sum of the shares
+    job_flops = bench.sum_over_ranks(1e12 * (rank + 1), dist, torch.device("cpu"))
+    out[rank] = (total, sparse, value, job_flops)
     dist.barrier()
     dist.destroy_process_group()
 
@@ -41,8 +43,8 @@ def test_two_ranks_aggregate_with_the_slowest_ranks_time():
         mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
         res = dict(out)
     assert res[0] == res[1]  # every rank ends with the same aggregate
-    total, sparse, value = res[0]
-    assert total == 15.0 and sparse == 6.0
+    total, sparse, value, job_flops = res[0]
+    assert total == 15.0 and sparse == 6.0 and job_flops == 3e12
     # 2 ranks x 3 calls x 1 TFLOP in 6 ms
     assert abs(value - 2 * 3 * 1.0 / 6e-3) < 1e-9
 
@@ -53,6 +55,7 @@ def test_single_rank_needs_no_process_group():
 
     assert bench.max_over_ranks([1.5, 2.5], None, torch.device("cpu")) == [1.5, 2.5]
     assert abs(bench.aggregate_tflops(2e12, 5, 10.0, 1) - 1000.0) < 1e-9
+    assert bench.sum_over_ranks(2.5, None, torch.device("cpu")) == 2.5
 
 
 def test_reference_arm_prints_on_rank_zero_only():
