@@ -1,30 +1,34 @@
 // Attention kernels of liblosa for sm_100a: dense attention, block-sparse attention over a
-// frozen CSR pattern (Eq. 4) and the exact block-mass pass (Eq. 1), as ONE warp-specialised
-// persistent kernel template.
+// frozen CSR pattern (Eq. 4), the exact block-mass pass (Eq. 1) and the fused construction step,
+// as ONE warp-specialised persistent kernel template with two thread layouts.
 //
-// CTA = 12 warps.  Warps 0-3 are utility warps: warp 0 is the TMA producer, which streams the
-// query tiles and the K / V tiles named by the tile list into 128B-swizzled shared-memory rings
-// (a K/V tile is 128 keys: 128 / C key blocks, one copy per block and 64-column slab); warps 1
-// and 2 (one elected thread each) issue the tcgen05 MMAs of query tile 0 and 1: S = Q K^T from
-// shared memory into TMEM, O += P V with P read from TMEM (bf16, written over S) and V from
-// shared memory as the MN-major operand; warp 3 publishes the tile list every other warp
-// follows (sparse mode: streamed from lists that build_tile_lists_kernel made before the
-// launch).  Warps 4-7 and 8-11 are two softmax warpgroups, each owning one 128-row query tile
-// (thread = query row = TMEM lane); they take their registers from the utility warpgroup.
+// Warps 0-3 are utility warps: warp 0 is the TMA producer, which streams the query tiles and the
+// K / V tiles named by the tile list into 128B-swizzled shared-memory rings (a K/V tile is 128
+// keys: 128 / C key blocks, one copy per block and 64-column slab); warps 1 and 2 (one elected
+// thread each) issue the tcgen05 MMAs: S = Q K^T from shared memory into TMEM, O += P V with P
+// read from TMEM (bf16, written over S) and V from shared memory as the MN-major operand; warp 3
+// publishes the tile list every other warp follows (sparse mode: streamed from lists that
+// build_tile_lists_kernel made before the launch).  The softmax warps follow: two warpgroups, one
+// 128-row query tile each and one thread per query row (mass pass, fused step, fallback), or four
+// warpgroups with two threads per query row (dense and sparse forward); they take their registers
+// from the utility warpgroup.
 //
-// A work item is a pair of consecutive query tiles of one (batch, head).  The key blocks the
-// pair visits are the ascending union of the index lists of its query blocks (two lists, four
-// when R = 64), so a K/V tile needed by both tiles is loaded once, and MMAs are issued only for
-// the query tiles that list one of its blocks.  The items of the last, partly filled wave of
-// the persistent grid are cut into parts of their lists, merged by merge_parts_kernel.
+// A work item is a pair of consecutive query tiles of one (batch, head) - of one problem, in a
+// batched launch.  The key blocks the pair visits are the union of the index lists of its query
+// blocks (two lists, four when R = 64), so a K/V tile needed by both tiles is loaded once, and
+// MMAs are issued only for the query tiles that list one of its blocks.  The items of the last,
+// partly filled wave of the persistent grid are cut into parts of their lists, merged by
+// merge_parts_kernel.
 //
-// One S = Q K^T covers a whole K/V tile (128-wide MMAs: an MMA costs its issuing thread ~70
-// cycles whatever its width, so wide MMAs are what keeps the issuer off the critical path).
-// TMEM then holds exactly S and O of both query tiles, P overwrites S, and per query tile the
-// steps S -> softmax -> O += P V -> next S form a serial chain.  The two tiles run that chain
-// half a period apart: one tile's MMAs execute while the other tile's softmax runs.  The
-// attention modes keep no running maximum: they exponentiate against a reference that moves
-// only when a tile's row sums leave the safe range (the result does not depend on it).
+// One S = Q K^T covers a whole K/V tile (128-wide MMAs).  At head dimension 128 TMEM holds exactly
+// S and O of both query tiles, P overwrites S, and per query tile the steps S -> softmax ->
+// O += P V -> next S form a serial chain; the two tiles run that chain half a period apart, one
+// issuer each, under a lock that keeps their bursts of MMAs from interleaving.  At head dimension
+// 64 a third S buffer fits and the tiles take the three buffers in turn (one issuer for all
+// S = Q K^T, one for all O += P V).  No mode keeps a running maximum on its common path: the
+// exponentials are taken against a reference that moves only when a tile's row sums leave the safe
+// range (one thread per row), or never within a work unit (two threads per row; units whose scores
+// outgrow it are recomputed by a second launch of the one-thread-per-row kernel).
 //
 // Every wait is bounded; a wait that expires raises the CTA's abort flag, records
 // LOSA_ERR_TIMEOUT, and all roles leave through the common teardown that frees TMEM.
@@ -163,6 +167,8 @@ struct Params {
   float* lse;
   int* work_counter;  // zeroed before the launch; CTAs draw work items from it
   float2* rowstat;  // mass modes: [grid][2][128] final (max, 1/sum) of every row of the item
+                    // (fused step, two threads per row: [grid][2][2][128] the halves' row sums)
+  float* rowinv;    // fused step, two threads per row: [grid][2][128] 1 / (row sum) of every row
   float2* table;  // mass modes: [grid][2][nKb][128] (sum of p, reference max) per row and key tile
   float scale_log2;
   int* status;
@@ -288,7 +294,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   using C = Cfg<D, R, C_, MODE, KT, SPLIT && D == 64>;
   using L = Lay<SPLIT>;
   using Ctl = Control<C::kNK, C::kNV, SPLIT, SPLIT && D == 64>;
-  static_assert(!SPLIT || (C::kHasV && !C::kWantMass), "two threads per row: attention-only modes");
+  static_assert(!SPLIT || C::kHasV, "two threads per row: the modes with an attention output");
   // Head dimension 64 leaves 128 tensor-memory columns unused (O takes 64 per query tile), enough
   // for a third score buffer.  The two query tiles then take the three buffers in turn, in the
   // order in which their S = Q K^T are issued, so that the S of a query tile's next key tile is
@@ -334,7 +340,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       ptx::mbar_init(&ctl->p_ready[i], L::kSoftmaxWarps / 2);  // one elected arrival per softmax warp
       ptx::mbar_init(&ctl->o_done[i], 1);
       ptx::mbar_init(&ctl->o_free[i], 128);  // the threads that read O out
-      ptx::mbar_init(&ctl->wg_bar[i], 128);
+      ptx::mbar_init(&ctl->wg_bar[i], 16 * L::kSoftmaxWarps);  // all softmax threads of a query tile
     }
     for (int i = 0; i < C::kNK; ++i) {
       ptx::mbar_init(&ctl->k_full[i], 1);
@@ -623,7 +629,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       // constant for every operand): 24 whole descriptors do not fit this warp's 72 registers
       // and spilled, which cost 4 % of the forward.  The mass pass has half as many operands,
       // and it and the fused mode were measured 3 % faster with whole descriptors.
-      constexpr bool kLoDesc = C::kHasV && !C::kWantMass;
+      constexpr bool kLoDesc = (C::kHasV && !C::kWantMass) || SPLIT;
       uint32_t qd[D / 16];
 #pragma unroll
       for (int kk = 0; kk < D / 16; ++kk)
@@ -1227,6 +1233,13 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     uint32_t tSrow = tmem_base + lane_base + qt * kSStride;
     uint32_t tS = tSrow + half * 64;
     const uint32_t tO = tmem_base + lane_base + (kRot ? 384 + qt * 64 : 256 + qt * 128);
+    // fused construction step: this row's column of the CTA's table of per-block sums of the
+    // unrounded exponentials, one float per row and 64-column half of a key tile when a key block
+    // fills the tile (the halves' entries are added at the end), else one per row and key block
+    float* const tabf = C::kWantMass ? reinterpret_cast<float*>(p.table) +
+                                           ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * 256 + row
+                                     : nullptr;
+    uint32_t nwg = 0;
     uint32_t kq = 0;  // rotating buffers: scores issued so far, counted as the issuer counts them
     uint32_t uses[3] = {0, 0, 0};  // ... and how many of them, per buffer, were this query tile's
     const int sub = (R == 64) ? (wl >> 1) : 0;
@@ -1247,7 +1260,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       void* const o_base = (p.problems != nullptr) ? p.problems[pbh / (p.B * p.H)].o : p.o;
       const int T = 2 * pr + qt;
       const int grow = T * 128 + row;
-      float m_ref = 0.f, l = 0.f;
+      float m_ref = 0.f, l = 0.f, le = 0.f;  // le: row sum of the unrounded exponentials (masses, LSE)
       bool have_ref = false, ovf = false;
       uint32_t pv_item = 0;
       for (;;) {
@@ -1354,6 +1367,9 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           // The output is normalised by the sum of the weights the tensor core multiplies with V -
           // P as rounded to bf16 - so that o is a weighted mean of V whatever the rounding does.
           float2 racc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+          float2 eacc[kHB];  // fused step: sums of the unrounded exponentials, per block of this half
+#pragma unroll
+          for (int i = 0; i < kHB; ++i) eacc[i] = make_float2(0.f, 0.f);
 #pragma unroll
           for (int c = 0; c < 64; c += 4) {
             if (whole && c == 32) ptx::tmem_wait_ld();
@@ -1370,17 +1386,30 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             sr[(c >> 1) + 1] = u1;
             racc[0] = ptx::add2(racc[0], ptx::unpack_bf16x2(u0));
             racc[1] = ptx::add2(racc[1], ptx::unpack_bf16x2(u1));
+            if (C::kWantMass) eacc[c / kBW] = ptx::add2(eacc[c / kBW], ptx::add2(x0, x1));
           }
           const float tsum = (racc[0].x + racc[0].y) + (racc[1].x + racc[1].y);
           ovf = ovf || __any_sync(0xffffffffu, !(tsum <= kSplitSafeSum));
           l += tsum;
           ptx::tmem_st32(tS, &sr[0]);
+          if (C::kWantMass) {
+#pragma unroll
+            for (int i = 0; i < kHB; ++i) {
+              const float es = eacc[i].x + eacc[i].y;
+              le += es;
+              const int g = (kG >= 2) ? half * kHB + i : 0;
+              const int64_t sb = (kG >= 2) ? (int64_t)(grp[g] & 0xffffu) : (int64_t)(grp[0] & 0xffffu) * 2 + half;
+              if (hv[i] > 0) tabf[sb * 128] = es;
+            }
+          }
         } else {
           // this half of the row lists none of the tile's keys: P = 0
           uint32_t z[32];
 #pragma unroll
           for (int c = 0; c < 32; ++c) z[c] = 0u;
           ptx::tmem_st32(tS, z);
+          // (a key block that fills the tile but ends before this half: its entry of the table is 0)
+          if (C::kWantMass && kG == 1 && pair_mine) tabf[((int64_t)(grp[0] & 0xffffu) * 2 + half) * 128] = 0.f;
         }
         ptx::tmem_wait_st();
         ++pv_item;
@@ -1393,12 +1422,21 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       // ---- end of the item: half 1 hands its row sums over, half 0 writes O / l
       // (two sets of slots, used by alternate items: half 1 may be an item ahead of half 0's read)
       float* const xset = ctl->xch + ((nitem & 1) * 2 + qt) * 128;
+      // (fused step: both halves need both sums; they go through the workspace, two sets as well)
+      float2* const gset = C::kWantMass ? p.rowstat + ((((int64_t)blockIdx.x * 2 + (nitem & 1)) * 2 + qt) * 2) * 128
+                                        : nullptr;
       ++nitem;
-      if (half == 1) xset[row] = l;
+      if (C::kWantMass) gset[half * 128 + row] = make_float2(le, l);
+      else if (half == 1) xset[row] = l;
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(pair_bar);
       LOSA_WAIT(pair_bar, npair & 1);
       ++npair;
+      if (C::kWantMass) {
+        const float2 other = gset[(half ^ 1) * 128 + row];
+        le += other.x;
+        l += other.y;
+      }
       if (ovf && lane == 0) {
         // (the pair's warps may both get here, and so may the other pairs: the unit is listed once)
         const int unit = partial ? p.split_first + (w - p.split_first) * p.split_parts + part : w;
@@ -1408,7 +1446,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
       }
       if (half == 0 && T < p.nQt) {
-        l += xset[row];
+        if (!C::kWantMass) l += xset[row];
         const bool valid = grow < p.N;
         const float inv = (l > 0.f) ? 1.f / l : 0.f;
         const int64_t off = (int64_t)b * p.sb + (int64_t)h * p.sh + (int64_t)grow * p.sn;
@@ -1462,6 +1500,58 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           ptx::tc_fence_before_sync();
           ptx::mbar_arrive(&ctl->o_free[qt]);
         }
+      }
+      if (C::kWantMass) {
+        // ---- fused construction step: the block masses of this query tile.  The reference did not
+        // move during the item, so a row's weight is 1 / (its sum of exponentials) and a mass is the
+        // mean over the query block's rows of weight x (the row's sum over the key block).
+        float* const inv_rows = p.rowinv + ((int64_t)blockIdx.x * 2 + qt) * 128;
+        if (half == 0 && T < p.nQt) {
+          const bool valid = grow < p.N;
+          inv_rows[row] = (valid && le > 0.f) ? 1.f / le : 0.f;
+          if (p.lse != nullptr && valid) p.lse[(int64_t)bh * p.N + grow] = (m_ref + log2f(le)) * kLn2;
+        }
+        ptx::mbar_arrive(&ctl->wg_bar[qt]);  // all eight warps of the query tile, with a bounded wait
+        LOSA_WAIT(&ctl->wg_bar[qt], nwg & 1);
+        ++nwg;
+        if (T < p.nQt) {
+          const float* tb = reinterpret_cast<const float*>(p.table) +
+                            ((int64_t)blockIdx.x * 2 + qt) * (int64_t)p.nKb * 256;
+          float iv[4];  // this lane's four rows
+#pragma unroll
+          for (int rr = 0; rr < 4; ++rr) iv[rr] = inv_rows[rr * 32 + lane];
+          for (int u = half * 4 + wl; u < p.nKb; u += 8) {
+            float acc[kQBT];
+#pragma unroll
+            for (int q = 0; q < kQBT; ++q) acc[q] = 0.f;
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr) {
+              const int r = rr * 32 + lane;
+              float wgt = 0.f;
+              if (iv[rr] > 0.f) {
+                const float sum = (kG >= 2) ? tb[(int64_t)u * 128 + r]
+                                            : tb[(int64_t)u * 256 + r] + tb[(int64_t)u * 256 + 128 + r];
+                wgt = sum * iv[rr];
+              }
+              acc[(rr * 32) / R] += wgt;
+            }
+#pragma unroll
+            for (int q = 0; q < kQBT; ++q) {
+              float a2 = acc[q];
+#pragma unroll
+              for (int d = 16; d > 0; d >>= 1) a2 += __shfl_xor_sync(0xffffffffu, a2, d);
+              const int g = T * kQBT + q;
+              if (lane == 0 && g < p.nQb) {
+                const int nvalid = min(R, p.N - g * R);
+                p.mass[((int64_t)bh * p.nQb + g) * p.nKb + u] = a2 / (float)nvalid;
+              }
+            }
+          }
+        }
+        // (the table and the row weights are written again by the next item)
+        ptx::mbar_arrive(&ctl->wg_bar[qt]);
+        LOSA_WAIT(&ctl->wg_bar[qt], nwg & 1);
+        ++nwg;
       }
     }
   }
@@ -1799,6 +1889,7 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
   prm.split_first = prm.nWork;
   prm.split_parts = 1;
   constexpr bool kAttnOnly = (MODE == kDense || MODE == kSparse);
+  constexpr bool kTwoPerRow = kAttnOnly || MODE == kFused;  // the modes that run with two threads per row
   if (kAttnOnly) {
     const int rest = (prm.nWork < ctas) ? prm.nWork : prm.nWork % ctas;
     int parts = rest > 0 ? ctas / rest : 1;
@@ -1815,9 +1906,9 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
     build_tile_lists_kernel<C::kNB, C::kG><<<prm.nUnits, 32, bm_bytes, st>>>(prm);
     LOSA_CUDA_TRY(cudaGetLastError());
   }
-  if constexpr (kAttnOnly) {
-    // The attention-only modes run with two threads per query row and a reference that never
-    // moves; the units whose scores outgrew it (none, on ordinary inputs) are listed, and a second
+  if constexpr (kTwoPerRow) {
+    // The modes with an attention output run with two threads per query row and a reference that
+    // never moves; the units whose scores outgrew it (none, on ordinary inputs) are listed, and a second
     // launch of the one-thread-per-row kernel, which returns at once when the list is empty,
     // recomputes them with a moving reference.
     prm.redo = 0;
@@ -1891,9 +1982,12 @@ size_t attn_workspace_bytes(AttnMode mode, const Geometry& g, int n_prob) {
     bytes += tl_count_bytes(g, n_prob);
     return bytes;
   }
-  // counter, per-CTA row statistics, per-CTA table of one entry per row and key tile
-  return kCounterBytes + kRowstatBytes +
-         (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2);
+  // counter, per-CTA row statistics (three times as many for the fused step with two threads per
+  // row: two sets of the halves' row sums, and the rows' weights), per-CTA table of one entry per
+  // row and key tile, and the fused step's list of units for the fallback launch
+  return kCounterBytes + (mode == kFused ? 5 : 1) * kRowstatBytes +
+         (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2) +
+         (mode == kFused ? tl_count_bytes(g, 1) : 0);
 }
 
 // Batched launch (n_prob > 1, attention-only modes): `layers` is a host array of n_prob problems of
@@ -1927,7 +2021,8 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
   prm.work_counter = static_cast<int*>(ws);
   prm.rowstat = reinterpret_cast<float2*>(static_cast<char*>(ws) + kCounterBytes);
   prm.table = reinterpret_cast<float2*>(static_cast<char*>(ws) + kCounterBytes +
-                                        ((mode == kMass || mode == kFused) ? kRowstatBytes : 0));
+                                        (mode == kFused ? 5 : mode == kMass ? 1 : 0) * kRowstatBytes);
+  prm.rowinv = reinterpret_cast<float*>(static_cast<char*>(ws) + kCounterBytes + 4 * kRowstatBytes);
   prm.part_ml = reinterpret_cast<float2*>(static_cast<char*>(ws) + kCounterBytes);
   prm.part_o = reinterpret_cast<float*>(static_cast<char*>(ws) + kCounterBytes + kPartMlBytes);
   {
@@ -1961,6 +2056,9 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
     prm.redo_list = reinterpret_cast<int*>(
         tl + (mode == kSparse ? tl_count_bytes(g, n_prob) + tl_entries_bytes(g, n_prob) : 0) +
         (n_prob > 1 ? (size_t)n_prob * sizeof(ProblemEntry) : 0));
+    if (mode == kFused)  // behind the table
+      prm.redo_list = reinterpret_cast<int*>(reinterpret_cast<char*>(prm.table) +
+                                             (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2));
   }
   prm.scale_log2 = g.scale * kLog2e;
   int rc = LOSA_OK;
