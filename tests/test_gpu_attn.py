@@ -490,3 +490,40 @@ def test_block_mass_with_one_key_far_above_the_reference(D, col):
     assert losa.losa_async_status() == 0
     assert np.abs(mass_f.cpu().numpy().reshape(ref.shape) - ref).max() <= util.MASS_TOL
     util.assert_output_close(o_f, orc.dense_attn(qn, kn, vn), "fused o with an outlier key")
+
+
+@pytest.mark.parametrize("D,BLK", [(128, 128), (64, 64)])
+def test_rows_that_outgrow_their_reference_in_whole_and_cut_work_units(D, BLK):
+    """The forward keeps, per work unit, the reference of the unit's first tile; a unit whose scores
+    rise far above it is handed to a second launch that moves the reference.  More work items than
+    SMs, so that some units are whole items and the last ones are parts; half of the heads carry
+    keys 60 nats above the rest from the third tile on, the other half do not (their units must
+    not be touched by the second launch: compared with the oracle all the same)."""
+    losa = lib()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    B, N = 1, 128 * 7 + 50
+    H = sms // 4 + 6                       # 4 pairs of query tiles per head: more items than SMs
+    assert H * 4 > sms
+    g = torch.Generator("cpu").manual_seed(77)
+    q = torch.randn(B, H, N, D, generator=g) * 0.3 + 1.0
+    k = torch.randn(B, H, N, D, generator=g) * 0.3
+    k[:, ::2, 300:] += 60.0 * (D ** 0.5) / D
+    v = torch.randn(B, H, N, D, generator=g)
+    q, k, v = q.bfloat16(), k.bfloat16(), v.bfloat16()
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    qn, kn, vn = util.to_np(q), util.to_np(k), util.to_np(v)
+    o = losa.losa_attn(qd, kd, vd, BLK, BLK, out_dtype=torch.float32)
+    assert losa.losa_async_status() == 0
+    util.assert_output_close(o, orc.dense_attn(qn, kn, vn), "dense, some heads outgrow the reference")
+    nb = -(-N // BLK)
+    off, idx = util.random_csr(B * H * nb, nb, 9, 0.7)
+    o_s = losa.losa_sparse_attn(qd, kd, vd, torch.from_numpy(off).cuda(), torch.from_numpy(idx).cuda(),
+                                BLK, BLK, out_dtype=torch.float32)
+    assert losa.losa_async_status() == 0
+    ref_s = orc.blocks_to_tokens(orc.sparse_attn(qn, kn, vn, BLK, BLK, off, idx), B, H, N)
+    util.assert_output_close(o_s, ref_s, "sparse, some heads outgrow the reference")
+    o_f, mass = losa.losa_attn_mass(qd, kd, vd, BLK, BLK, out_dtype=torch.float32)
+    assert losa.losa_async_status() == 0
+    util.assert_output_close(o_f, orc.dense_attn(qn, kn, vn), "fused, some heads outgrow the reference")
+    ref_m = orc.block_mass(qn, kn, BLK, BLK)
+    assert np.abs(mass.cpu().numpy().reshape(ref_m.shape) - ref_m).max() <= util.MASS_TOL
