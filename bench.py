@@ -61,13 +61,12 @@ def merge_kernel_runs(wl) -> bool:
 
 
 def launches_per_step(wl, draws: int) -> int:
-    """Kernels of the library launched by one step: mass 1; select 3; every sparse call its tile-list
-    pre-pass, the attention kernel and the fallback kernel behind it (which returns at once when no
-    row outgrew its reference), plus the merge kernel when the last wave is cut into parts; the
-    dense call the same without the pre-pass; the fused construction step its kernel and the fallback
-    kernel behind it."""
+    """Kernels of the library launched by one step.  Every attention-shaped call launches its kernel
+    and the fallback kernel behind it (which returns at once when no row outgrew its reference): the
+    mass pass 2; select 3; every sparse call also its tile-list pre-pass, plus the merge kernel when the
+    last wave is cut into parts; the dense call the same without the pre-pass; the fused step 2."""
     merge = int(merge_kernel_runs(wl))
-    return 1 + 3 + draws * (3 + merge) + (2 + merge) + 2
+    return 2 + 3 + draws * (3 + merge) + (2 + merge) + 2
 
 
 def cpu_model() -> str:

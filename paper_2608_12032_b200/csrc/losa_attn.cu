@@ -291,10 +291,9 @@ template <int D, int R, int C_, int MODE, int KT, bool SPLIT>
 __global__ void __launch_bounds__(Lay<SPLIT>::kThreads, 1)
 losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, const Params p) {
-  using C = Cfg<D, R, C_, MODE, KT, SPLIT && D == 64>;
+  using C = Cfg<D, R, C_, MODE, KT, SPLIT && D == 64 && MODE != kMass>;
   using L = Lay<SPLIT>;
-  using Ctl = Control<C::kNK, C::kNV, SPLIT, SPLIT && D == 64>;
-  static_assert(!SPLIT || C::kHasV, "two threads per row: the modes with an attention output");
+  using Ctl = Control<C::kNK, C::kNV, SPLIT, SPLIT && D == 64 && MODE != kMass>;
   // Head dimension 64 leaves 128 tensor-memory columns unused (O takes 64 per query tile), enough
   // for a third score buffer.  The two query tiles then take the three buffers in turn, in the
   // order in which their S = Q K^T are issued, so that the S of a query tile's next key tile is
@@ -302,7 +301,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   // the tensor core.  One issuer warp issues every S = Q K^T of the CTA in that fixed order, the
   // other every O += P V; a buffer is written again only after the product that read its P has
   // completed (a barrier between the two issuers).
-  constexpr bool kRot = SPLIT && D == 64;
+  constexpr bool kRot = SPLIT && D == 64 && C::kHasV;
   constexpr int kC = C::kC, kG = C::kG, kQBT = C::kQBT, kNB = C::kNB, kW = C::kW, kNS = C::kNS;
   constexpr uint32_t kSStride = C::kSStride, kNVs = C::kNV > 0 ? C::kNV : 1;
   constexpr uint32_t kQMask = (1u << kQBT) - 1u;
@@ -335,7 +334,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       ptx::mbar_init(&ctl->q_empty[i], 1);
       for (int u = 0; u < 2; ++u) {
         ptx::mbar_init(&ctl->s_full[i][u], 1);
-        ptx::mbar_init(&ctl->s_free[i][u], 4);  // one elected arrival per softmax warp
+        ptx::mbar_init(&ctl->s_free[i][u], L::kSoftmaxWarps / 2);  // one elected arrival per softmax warp
       }
       ptx::mbar_init(&ctl->p_ready[i], L::kSoftmaxWarps / 2);  // one elected arrival per softmax warp
       ptx::mbar_init(&ctl->o_done[i], 1);
@@ -1309,7 +1308,13 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         } else {
           if (((memb >> (qt * kQBT)) & kQMask) == 0) continue;
           // S of this key tile is complete, and so is every earlier product into O
-          LOSA_WAIT(&ctl->s_full[qt][0], nsub & 1);
+          // (the mass pass has two S buffers per query tile and no O)
+          const uint32_t buf = nsub % kNS;
+          if (!C::kHasV) {
+            tSrow = tmem_base + lane_base + qt * kSStride + buf * 128;
+            tS = tSrow + half * 64;
+          }
+          LOSA_WAIT(&ctl->s_full[qt][buf], (nsub / kNS) & 1);
         }
         ptx::tc_fence_after_sync();
         if (!have_ref && pair_mine) {
@@ -1356,6 +1361,13 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 if ((c % kBW) >= hv[c / kBW]) sr[c] = 0xff800000u;
             }
           }
+          if (!C::kHasV) {
+            // mass pass: the scores are in registers and nothing is packed over them: the buffer goes back
+            ptx::tmem_wait_ld();
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&ctl->s_free[qt][nsub % kNS]);
+          }
           // key blocks the row's query block does not list get -inf as the addend of the scaling FMA
           const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
           float2 nm2[kHB];
@@ -1372,7 +1384,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           for (int i = 0; i < kHB; ++i) eacc[i] = make_float2(0.f, 0.f);
 #pragma unroll
           for (int c = 0; c < 64; c += 4) {
-            if (whole && c == 32) ptx::tmem_wait_ld();
+            if (C::kHasV && whole && c == 32) ptx::tmem_wait_ld();
             float2 x0 = ptx::fma2(
                 make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nm2[c / kBW]);
             float2 x1 = ptx::fma2(
@@ -1381,17 +1393,23 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             x0.y = ptx::ex2_approx(x0.y);
             x1.x = ptx::ex2_approx(x1.x);
             x1.y = ptx::ex2_approx(x1.y);
-            const uint32_t u0 = ptx::pack_bf16x2(x0.x, x0.y), u1 = ptx::pack_bf16x2(x1.x, x1.y);
-            sr[c >> 1] = u0;
-            sr[(c >> 1) + 1] = u1;
-            racc[0] = ptx::add2(racc[0], ptx::unpack_bf16x2(u0));
-            racc[1] = ptx::add2(racc[1], ptx::unpack_bf16x2(u1));
+            if (C::kHasV) {
+              const uint32_t u0 = ptx::pack_bf16x2(x0.x, x0.y), u1 = ptx::pack_bf16x2(x1.x, x1.y);
+              sr[c >> 1] = u0;
+              sr[(c >> 1) + 1] = u1;
+              racc[0] = ptx::add2(racc[0], ptx::unpack_bf16x2(u0));
+              racc[1] = ptx::add2(racc[1], ptx::unpack_bf16x2(u1));
+            }
             if (C::kWantMass) eacc[c / kBW] = ptx::add2(eacc[c / kBW], ptx::add2(x0, x1));
           }
-          const float tsum = (racc[0].x + racc[0].y) + (racc[1].x + racc[1].y);
+          float tsum = (racc[0].x + racc[0].y) + (racc[1].x + racc[1].y);
+          if (!C::kHasV) {
+#pragma unroll
+            for (int i = 0; i < kHB; ++i) tsum += eacc[i].x + eacc[i].y;
+          }
           ovf = ovf || __any_sync(0xffffffffu, !(tsum <= kSplitSafeSum));
           l += tsum;
-          ptx::tmem_st32(tS, &sr[0]);
+          if (C::kHasV) ptx::tmem_st32(tS, &sr[0]);
           if (C::kWantMass) {
 #pragma unroll
             for (int i = 0; i < kHB; ++i) {
@@ -1404,18 +1422,27 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
         } else {
           // this half of the row lists none of the tile's keys: P = 0
-          uint32_t z[32];
+          if (C::kHasV) {
+            uint32_t z[32];
 #pragma unroll
-          for (int c = 0; c < 32; ++c) z[c] = 0u;
-          ptx::tmem_st32(tS, z);
+            for (int c = 0; c < 32; ++c) z[c] = 0u;
+            ptx::tmem_st32(tS, z);
+          } else {
+            // mass pass: the buffer goes back untouched
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&ctl->s_free[qt][nsub % kNS]);
+          }
           // (a key block that fills the tile but ends before this half: its entry of the table is 0)
           if (C::kWantMass && kG == 1 && pair_mine) tabf[((int64_t)(grp[0] & 0xffffu) * 2 + half) * 128] = 0.f;
         }
-        ptx::tmem_wait_st();
-        ++pv_item;
-        ptx::tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(kRot ? &ctl->rot_p_ready[qt * 3 + rot_b] : &ctl->p_ready[qt]);
+        if (C::kHasV) {
+          ptx::tmem_wait_st();
+          ++pv_item;
+          ptx::tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(kRot ? &ctl->rot_p_ready[qt * 3 + rot_b] : &ctl->p_ready[qt]);
+        }
         ++nsub;
       }
 
@@ -1445,7 +1472,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if (slot < p.nUnits) p.redo_list[slot] = unit;
         }
       }
-      if (half == 0 && T < p.nQt) {
+      if (C::kHasV && half == 0 && T < p.nQt) {
         if (!C::kWantMass) l += xset[row];
         const bool valid = grow < p.N;
         const float inv = (l > 0.f) ? 1.f / l : 0.f;
@@ -1840,9 +1867,9 @@ int make_map(CUtensorMap* m, const void* base, const Geometry& g, int box_rows) 
 template <int D, int R, int C_, int MODE, int KT, bool SPLIT>
 int launch_kernel(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                   const Params& prm, int grid, cudaStream_t st) {
-  using C = Cfg<D, R, C_, MODE, KT, SPLIT && D == 64>;
+  using C = Cfg<D, R, C_, MODE, KT, SPLIT && D == 64 && MODE != kMass>;
   using L = Lay<SPLIT>;
-  using Ctl = Control<C::kNK, C::kNV, SPLIT, SPLIT && D == 64>;
+  using Ctl = Control<C::kNK, C::kNV, SPLIT, SPLIT && D == 64 && MODE != kMass>;
   // (one thread per row: 1024 bytes of slack to align the tiles; two threads per row: none left,
   // the kernel checks the alignment of its shared memory instead)
   const size_t smem = (SPLIT ? 0 : 1024) + 2 * C::kQBytes +
@@ -1889,7 +1916,7 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
   prm.split_first = prm.nWork;
   prm.split_parts = 1;
   constexpr bool kAttnOnly = (MODE == kDense || MODE == kSparse);
-  constexpr bool kTwoPerRow = kAttnOnly || MODE == kFused;  // the modes that run with two threads per row
+  constexpr bool kTwoPerRow = true;  // every mode runs with two threads per row; one per row is the fallback
   if (kAttnOnly) {
     const int rest = (prm.nWork < ctas) ? prm.nWork : prm.nWork % ctas;
     int parts = rest > 0 ? ctas / rest : 1;
@@ -1985,9 +2012,8 @@ size_t attn_workspace_bytes(AttnMode mode, const Geometry& g, int n_prob) {
   // counter, per-CTA row statistics (three times as many for the fused step with two threads per
   // row: two sets of the halves' row sums, and the rows' weights), per-CTA table of one entry per
   // row and key tile, and the fused step's list of units for the fallback launch
-  return kCounterBytes + (mode == kFused ? 5 : 1) * kRowstatBytes +
-         (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2) +
-         (mode == kFused ? tl_count_bytes(g, 1) : 0);
+  return kCounterBytes + 5 * kRowstatBytes +
+         (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2) + tl_count_bytes(g, 1);
 }
 
 // Batched launch (n_prob > 1, attention-only modes): `layers` is a host array of n_prob problems of
@@ -2021,7 +2047,7 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
   prm.work_counter = static_cast<int*>(ws);
   prm.rowstat = reinterpret_cast<float2*>(static_cast<char*>(ws) + kCounterBytes);
   prm.table = reinterpret_cast<float2*>(static_cast<char*>(ws) + kCounterBytes +
-                                        (mode == kFused ? 5 : mode == kMass ? 1 : 0) * kRowstatBytes);
+                                        ((mode == kFused || mode == kMass) ? 5 : 0) * kRowstatBytes);
   prm.rowinv = reinterpret_cast<float*>(static_cast<char*>(ws) + kCounterBytes + 4 * kRowstatBytes);
   prm.part_ml = reinterpret_cast<float2*>(static_cast<char*>(ws) + kCounterBytes);
   prm.part_o = reinterpret_cast<float*>(static_cast<char*>(ws) + kCounterBytes + kPartMlBytes);
@@ -2056,7 +2082,7 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
     prm.redo_list = reinterpret_cast<int*>(
         tl + (mode == kSparse ? tl_count_bytes(g, n_prob) + tl_entries_bytes(g, n_prob) : 0) +
         (n_prob > 1 ? (size_t)n_prob * sizeof(ProblemEntry) : 0));
-    if (mode == kFused)  // behind the table
+    if (mode == kFused || mode == kMass)  // behind the table
       prm.redo_list = reinterpret_cast<int*>(reinterpret_cast<char*>(prm.table) +
                                              (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2));
   }
