@@ -100,9 +100,10 @@ size_t losa_workspace_bytes(int op, const losa_problem_t* p);
  * i.e. the paper's M(i,j) divided by the number of valid rows of query block i, so
  * that each row of `mass` sums to 1 and Eq. 3's threshold theta*R becomes tau.
  * One pass over Q K^T: every row keeps a running sum of exponentials against a reference
- * score that is raised whenever a tile's sums leave the safe range (for C < 128 the running
- * maximum itself); the per-key-block sums are taken in the same pass and normalised by the
- * row's final sum at the end.
+ * score (the row's maximum over its first key tile; rows whose later scores outgrow the
+ * fp32 range around it are recomputed with a running maximum by a second launch on the same
+ * stream); the per-key-block sums are taken in the same pass and normalised by the row's
+ * final sum at the end.
  *   q, k    bf16 [B,H,N,D] (strides from p)
  *   mass    f32  [B,H,nQb,nKb] contiguous, fully overwritten
  *   lse     f32  [B,H,N] contiguous or NULL: natural-log sum-exp of each row's scaled scores
@@ -183,12 +184,17 @@ int losa_select_noalloc(int32_t B, int32_t H, int32_t nQb, int32_t nKb, const fl
  * The CSR must satisfy losa_validate_csr(); a block index outside [0, nKb) is skipped and
  * reported as LOSA_ERR_BAD_INDEX, never dereferenced.
  *   q, k, v  bf16 [B,H,N,D];  o  [B,H,N,D] with the same strides, bf16 or f32 (o_dtype)
- *   ws       >= losa_workspace_bytes(LOSA_OP_SPARSE_ATTN, p) bytes (about 21 MB at D = 128:
- *            the counter the persistent CTAs draw work items from, and the partial results
- *            of the last work items, which are processed in parts and merged by a second
- *            kernel on the same stream); not shared between calls that may run
+ *   ws       >= losa_workspace_bytes(LOSA_OP_SPARSE_ATTN, p) bytes (about 21 MB at D = 128
+ *            plus the work units' tile lists: the counter the persistent CTAs draw work
+ *            items from, the partial results of the last work items, which are processed in
+ *            parts and merged by a second kernel on the same stream, and the list of work
+ *            units that a fallback launch recomputes because their scores outgrew the
+ *            reference of their first tile); not shared between calls that may run
  *            concurrently; contents undefined afterwards.  The result does not depend on
- *            timing: the same call on the same GPU gives the same bits.                   */
+ *            timing: the same call on the same GPU gives the same bits.
+ * The output is normalised by the sum of the bf16-rounded weights the tensor core multiplies
+ * with V, so every output row is a weighted mean of value rows (exact for a row that a
+ * single key dominates).                                                                 */
 int losa_sparse_attn(const losa_problem_t* p, const void* q, const void* k, const void* v,
                      const int32_t* offsets, const int32_t* kv_idx, void* o, int o_dtype,
                      void* ws, size_t ws_bytes, void* cuda_stream);
