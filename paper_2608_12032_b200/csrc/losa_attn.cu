@@ -37,6 +37,7 @@
 #include <math.h>
 
 #include <atomic>
+#include <cstddef>
 #include <vector>
 
 #include "losa_common.cuh"
@@ -44,6 +45,10 @@
 
 namespace losa {
 namespace {
+
+#ifndef LOSA_USE_PAIR
+#define LOSA_USE_PAIR 1
+#endif
 
 std::atomic<uint32_t> g_stall_polls{0u};  // > 0: the next attention launch is a diagnostic one
 
@@ -136,6 +141,7 @@ struct Cfg {
 // lives in the workspace and is written by the host before the launch.
 struct alignas(128) ProblemEntry {
   CUtensorMap map_q, map_k, map_v;
+  CUtensorMap map_kh;  // K with boxes of at most 64 keys (the CTA-pair kernel copies half a K tile per CTA)
   void* o;
   const int32_t* offsets;
   const int32_t* kv_idx;
@@ -1607,6 +1613,8 @@ teardown:
   }
 }
 
+#include "losa_attn_pair.cuh"
+
 #undef LOSA_TL_PUT_BULK
 #undef LOSA_TL_NEXT_TILE
 #undef LOSA_TL_NEXT
@@ -1898,6 +1906,55 @@ int launch_kernel(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMa
   return LOSA_OK;
 }
 
+// Configures (once per device) and launches the CTA-pair kernel on `clusters` pairs; *max_clusters
+// (if not null) receives how many pairs the device can hold at once.
+template <int C_, int MODE>
+int launch_pair(const CUtensorMap& mq, const CUtensorMap& mkh, const CUtensorMap& mv, const Params& prm,
+                int clusters, cudaStream_t st, int* max_clusters) {
+  using L = Lay<true>;
+  constexpr size_t smem = kPairQBytes + (size_t)(kPairNK + kPairNV) * kPairStage + sizeof(PairControl);
+  static_assert(smem <= 227 * 1024, "shared memory of one CTA");
+  auto kern = losa_pair_kernel<C_, MODE>;
+  static int max_on[kMaxDevices] = {};
+  int dev = 0;
+  LOSA_CUDA_TRY(cudaGetDevice(&dev));
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.blockDim = dim3(L::kThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (max_on[dev] == 0) {
+    cudaFuncAttributes fa;
+    LOSA_CUDA_TRY(cudaFuncGetAttributes(&fa, kern));
+    if (fa.numRegs * L::kThreads < 128 * L::kRegsUtility + 32 * L::kSoftmaxWarps * L::kRegsSoftmax) {
+      set_cuda_error(cudaErrorLaunchOutOfResources, "register budget of losa_pair_kernel");
+      return LOSA_ERR_UNSUPPORTED;
+    }
+    LOSA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    cfg.gridDim = dim3(2 * kMaxPersistentCtas, 1, 1);
+    int n = 0;
+    LOSA_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, kern, &cfg));
+    if (n < 1) {
+      set_cuda_error(cudaErrorLaunchOutOfResources, "no resident CTA pair of losa_pair_kernel");
+      return LOSA_ERR_UNSUPPORTED;
+    }
+    max_on[dev] = n;
+  }
+  if (max_clusters != nullptr) {
+    *max_clusters = max_on[dev];
+    return LOSA_OK;
+  }
+  cfg.gridDim = dim3(2 * clusters, 1, 1);
+  LOSA_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, mq, mkh, mv, prm));
+  return LOSA_OK;
+}
+
 template <int D, int R, int C_, int MODE, int KT>
 int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Params prm, int sms,
              cudaStream_t st) {
@@ -1907,7 +1964,23 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
   if ((rc = make_map(&mq, q, g, 128)) != LOSA_OK) return rc;
   if ((rc = make_map(&mk, k, g, C::kC)) != LOSA_OK) return rc;
   if ((rc = make_map(&mv, C::kHasV ? v : k, g, C::kC)) != LOSA_OK) return rc;
-  const int ctas = min(sms, kMaxPersistentCtas);
+  int ctas = min(sms, kMaxPersistentCtas);
+  // Head dimension 128 with 128-row query blocks and key blocks of 64 or 128, attention output
+  // only: pairs of CTAs, one work item per pair at a time (see losa_attn_pair.cuh); the single-CTA
+  // kernels stay the fallback.  (With 32-key blocks the pair kernel was measured slower than the
+  // single-CTA kernel, 6.3 against 5.9 ms for the dense forward at the Wan shape, and is not used.)
+  constexpr bool kPairMode =
+      LOSA_USE_PAIR && D == 128 && R == 128 && C_ >= 64 && (MODE == kDense || MODE == kSparse);
+  bool pair = false;  // (a device that cannot hold a pair of these CTAs runs the single-CTA kernel)
+  CUtensorMap mkh;
+  if constexpr (kPairMode) {
+    if ((rc = make_map(&mkh, k, g, C::kC < 64 ? C::kC : 64)) != LOSA_OK) return rc;
+    int fit = 0;
+    if (launch_pair<C_, MODE>(mq, mkh, mv, prm, 0, st, &fit) == LOSA_OK && fit >= 1 && sms >= 2) {
+      pair = true;
+      ctas = min(min(sms / 2, fit), kMaxPersistentCtas);
+    }
+  }
   // The items of the last, partly filled wave of the persistent grid (all items, if there are
   // fewer than CTAs) are cut into parts of the key range, so that the wave ends after 1/parts of
   // an item; their partial results are merged by a second, small kernel.  Attention output
@@ -1939,11 +2012,22 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
     // launch of the one-thread-per-row kernel, which returns at once when the list is empty,
     // recomputes them with a moving reference.
     prm.redo = 0;
-    if ((rc = launch_kernel<D, R, C_, MODE, KT, true>(mq, mk, mv, prm, grid, st)) != LOSA_OK) return rc;
+    bool launched = false;
+    if constexpr (kPairMode) {
+      if (pair) {
+        if ((rc = launch_pair<C_, MODE>(mq, mkh, mv, prm, grid, st, nullptr)) != LOSA_OK) return rc;
+        launched = true;
+      }
+    }
+    if (!launched) {
+      if ((rc = launch_kernel<D, R, C_, MODE, KT, true>(mq, mk, mv, prm, grid, st)) != LOSA_OK) return rc;
+    }
     if (!prm.stall) {
       prm.redo = 1;
       prm.work_counter += 2;  // its own counter (zeroed with the first)
-      if ((rc = launch_kernel<D, R, C_, MODE, KT, false>(mq, mk, mv, prm, grid, st)) != LOSA_OK) return rc;
+      // (as many CTAs as SMs, whichever kernel ran first)
+      const int rgrid = min(min(sms, kMaxPersistentCtas), prm.nUnits);
+      if ((rc = launch_kernel<D, R, C_, MODE, KT, false>(mq, mk, mv, prm, rgrid, st)) != LOSA_OK) return rc;
     }
   } else {
     prm.redo = 0;
@@ -2005,8 +2089,8 @@ size_t attn_workspace_bytes(AttnMode mode, const Geometry& g, int n_prob) {
     if (mode == kSparse) bytes += tl_count_bytes(g, n_prob) + tl_entries_bytes(g, n_prob);
     // batched launch: the table of the problems' tensor maps and pointers
     if (n_prob > 1) bytes += (size_t)n_prob * sizeof(ProblemEntry);
-    // the work units handed to the fallback launch
-    bytes += tl_count_bytes(g, n_prob);
+    // the work units handed to the fallback launch (each CTA of a pair may list a unit)
+    bytes += 2 * tl_count_bytes(g, n_prob);
     return bytes;
   }
   // counter, per-CTA row statistics (three times as many for the fused step with two threads per
@@ -2065,6 +2149,7 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
         if ((rc = make_map(&host[i].map_q, layers[i].q, g, 128)) != LOSA_OK) return rc;
         if ((rc = make_map(&host[i].map_k, layers[i].k, g, g.C)) != LOSA_OK) return rc;
         if ((rc = make_map(&host[i].map_v, layers[i].v, g, g.C)) != LOSA_OK) return rc;
+        if ((rc = make_map(&host[i].map_kh, layers[i].k, g, g.C < 64 ? g.C : 64)) != LOSA_OK) return rc;
         host[i].o = layers[i].o;
         host[i].offsets = layers[i].offsets;
         host[i].kv_idx = layers[i].kv_idx;

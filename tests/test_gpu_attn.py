@@ -166,8 +166,10 @@ def test_chain_mass_select_sparse_on_named_workloads(name, taus):
 def test_two_guidance_branches_in_one_batch_keep_their_own_patterns():
     """The two classifier-free-guidance branches travel as B = 2 and each (b, h, query block) row
     of the CSR is its own pattern: one batched pass over both branches must equal the two
-    single-branch passes bit for bit (masses, CSR, output), and each branch must match the oracle
-    on its own pattern.  The branches get differently sharp scores, so their patterns differ."""
+    single-branch passes bit for bit in masses and CSR, and in the output up to the rounding of P
+    (a launch with fewer work units cuts them into more parts, each with its own reference, so the
+    bf16 weights round differently), and each branch must match the oracle on its own pattern.
+    The branches get differently sharp scores, so their patterns differ."""
     losa = lib()
     H, N, D, BLK, tau = 2, 900, 128, 128, 0.9
     q0, k0, v0 = make(1, H, N, D, 71, 1.0)
@@ -191,7 +193,7 @@ def test_two_guidance_branches_in_one_batch_keep_their_own_patterns():
         lo, hi = off_h[b * rows], off_h[(b + 1) * rows]
         assert np.array_equal(ob_.cpu().numpy(), off_h[b * rows:(b + 1) * rows + 1] - lo)
         assert np.array_equal(ib_.cpu().numpy()[: hi - lo], idx_h[lo:hi])
-        assert torch.equal(o_b[0], o[b])
+        assert (o_b[0] - o[b]).abs().max().item() <= util.MAX_ABS_TOL
         per_branch.append(util.csr_rows(ob_.cpu().numpy(), ib_.cpu().numpy()[: hi - lo]))
         # against the oracle, branch by branch
         qn, kn, vn = (util.to_np(t[b:b + 1]) for t in (q, k, v))
