@@ -45,7 +45,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one sparse-forward launch, from an ncu capture of
 # the same kernel on the same workload (a profiler run: not re-measured by this script, which never
 # runs under a profiler); None where no capture was taken
-NCU_DRAM_BYTES_PER_LAUNCH = {"wan": 0.303693e9 + 0.082910e9}
+NCU_DRAM_BYTES_PER_LAUNCH = {"wan": 0.303407e9 + 0.082542e9}
 NCU_TRAFFIC_SOURCE = "ncu capture of the sparse forward at the Wan2.1 shape (dram__bytes_read.sum + dram__bytes_write.sum)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -54,6 +54,8 @@ def merge_kernel_runs(wl) -> bool:
     """Whether the attention-only calls launch their merge kernel for this shape: the host rule of
     the library, restated (work items = pairs of 128-row query tiles per head)."""
     ctas = min(torch.cuda.get_device_properties(0).multi_processor_count, 160)
+    if wl.D == 128 and wl.R == 128 and wl.C >= 64:
+        ctas //= 2  # these shapes run on pairs of CTAs: one work item per pair at a time
     n_work = wl.B * wl.H * ((-(-wl.N // 128) + 1) // 2)
     rest = n_work if n_work < ctas else n_work % ctas
     parts = min(ctas // rest, 8, -(-wl.N // wl.C)) if rest else 1
