@@ -131,7 +131,7 @@ class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
     def __init__(self, index: int):
-        self.samples, self.reasons = [], set()
+        self.samples, self.power, self.reasons = [], [], set()
         self.max_mhz = None
         self._stop = threading.Event()
         self._thread = None
@@ -157,6 +157,10 @@ class ClockSampler:
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
                 try:
+                    self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+                except Exception:
+                    pass
+                try:
                     mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
                 except Exception:
                     mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
@@ -165,7 +169,7 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            time.sleep(0.05)
+            time.sleep(0.01)
 
     def __enter__(self):
         if self.nv is not None:
@@ -184,6 +188,8 @@ class ClockSampler:
             "sm_max_mhz": self.max_mhz,
             "reasons": sorted(self.reasons),
             "samples": len(self.samples),
+            "sm_min_mhz": min(self.samples) if self.samples else None,
+            "power_w": statistics.median(self.power) if self.power else None,
         }
 
 

@@ -16,6 +16,9 @@ NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC,
 ]
+# extra compiler flags for measurement builds, e.g. LOSA_NVCC_EXTRA=-DLOSA_USE_PAIR=0 (the forward
+# at head dimension 128 on single CTAs instead of pairs); use with --force
+NVCC_FLAGS += os.environ.get("LOSA_NVCC_EXTRA", "").split()
 
 
 def _nvcc() -> str:
