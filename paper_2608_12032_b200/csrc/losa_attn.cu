@@ -32,6 +32,11 @@
 //
 // Every wait is bounded; a wait that expires raises the CTA's abort flag, records
 // LOSA_ERR_TIMEOUT, and all roles leave through the common teardown that frees TMEM.
+//
+// The dense and sparse forward at head dimension 128 with 128-row query blocks and key blocks of 64
+// or 128 keys run in a second kernel, losa_pair_kernel (losa_attn_pair.cuh, included below): pairs
+// of CTAs that multiply together (tcgen05.mma.cta_group::2), one query tile and three S buffers per
+// CTA.  This kernel serves every other shape and mode and the fallback launch of all of them.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <math.h>
@@ -1045,8 +1050,8 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 const uint32_t u0 = ptx::pack_bf16x2(x0.x, x0.y), u1 = ptx::pack_bf16x2(x1.x, x1.y);
                 sr[c >> 1] = u0;
                 sr[(c >> 1) + 1] = u1;
-                racc[0] = ptx::add2(racc[0], ptx::unpack_bf16x2(u0));
-                racc[1] = ptx::add2(racc[1], ptx::unpack_bf16x2(u1));
+                ptx::add_bf16x2(racc[0], u0);
+                ptx::add_bf16x2(racc[1], u1);
               }
             }
             tsum = 0.f;
@@ -1403,8 +1408,8 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               const uint32_t u0 = ptx::pack_bf16x2(x0.x, x0.y), u1 = ptx::pack_bf16x2(x1.x, x1.y);
               sr[c >> 1] = u0;
               sr[(c >> 1) + 1] = u1;
-              racc[0] = ptx::add2(racc[0], ptx::unpack_bf16x2(u0));
-              racc[1] = ptx::add2(racc[1], ptx::unpack_bf16x2(u1));
+              ptx::add_bf16x2(racc[0], u0);
+              ptx::add_bf16x2(racc[1], u1);
             }
             if (C::kWantMass) eacc[c / kBW] = ptx::add2(eacc[c / kBW], ptx::add2(x0, x1));
           }

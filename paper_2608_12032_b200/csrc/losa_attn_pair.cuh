@@ -614,8 +614,8 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const uint32_t u0 = ptx::pack_bf16x2(x0.x, x0.y), u1 = ptx::pack_bf16x2(x1.x, x1.y);
             sr[c >> 1] = u0;
             sr[(c >> 1) + 1] = u1;
-            racc[0] = ptx::add2(racc[0], ptx::unpack_bf16x2(u0));
-            racc[1] = ptx::add2(racc[1], ptx::unpack_bf16x2(u1));
+            ptx::add_bf16x2(racc[0], u0);
+            ptx::add_bf16x2(racc[1], u1);
           }
           const float tsum = (racc[0].x + racc[0].y) + (racc[1].x + racc[1].y);
           ovf = ovf || __any_sync(0xffffffffu, !(tsum <= kSplitSafeSum));
