@@ -45,7 +45,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one sparse-forward launch, from an ncu capture of
 # the same kernel on the same workload (a profiler run: not re-measured by this script, which never
 # runs under a profiler); None where no capture was taken
-NCU_DRAM_BYTES_PER_LAUNCH = {"wan": 0.303407e9 + 0.082542e9}
+NCU_DRAM_BYTES_PER_LAUNCH = {"wan": 0.303640e9 + 0.082585e9}
 NCU_TRAFFIC_SOURCE = "ncu capture of the sparse forward at the Wan2.1 shape (dram__bytes_read.sum + dram__bytes_write.sum)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
