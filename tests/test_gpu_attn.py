@@ -114,6 +114,7 @@ def test_fused_construction_step_matches_oracle_and_the_separate_calls(shape):
     # range and merge them, which changes the summation order, not the result beyond rounding: two
     # approximations, each within the tolerance of the exact result
     assert (o - o_sep).abs().max().item() <= 2 * util.MAX_ABS_TOL
+    assert (o - o_sep).abs().mean().item() <= 2 * util.MEAN_ABS_TOL  # no systematic difference
     ref, ref_lse = orc.block_mass(qn, kn, BLK, BLK, return_lse=True)
     got = mass.cpu().numpy().reshape(ref.shape).astype(np.float64)
     assert np.abs(got - ref).max() <= util.MASS_TOL

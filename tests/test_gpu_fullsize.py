@@ -154,6 +154,9 @@ def test_full_size_parity_on_sampled_query_blocks(name, per_head):
         # two approximations of the same values (the attention-only call also cuts its last work items
         # into parts and merges them): each is within the tolerance of the exact result
         assert (o_f - o_d).abs().max().item() <= 2 * util.MAX_ABS_TOL
+        assert (o_f - o_d).abs().mean().item() <= 2 * util.MEAN_ABS_TOL  # no systematic difference
+        record["fused_vs_dense_max_abs"] = (o_f - o_d).abs().max().item()
+        record["fused_vs_dense_mean_abs"] = (o_f - o_d).abs().mean().item()
         gmf = mass_f.cpu().numpy().reshape(wl.rows, wl.nKb)
         assert float(np.abs(gmf[ids] - ref_mass).max()) <= util.MASS_TOL
         assert np.abs(gmf.astype(np.float64).sum(1) - 1.0).max() <= util.MASS_TOL
