@@ -54,6 +54,9 @@ namespace {
 #ifndef LOSA_USE_PAIR
 #define LOSA_USE_PAIR 1
 #endif
+#ifndef LOSA_PAIR_FUSED
+#define LOSA_PAIR_FUSED 1
+#endif
 
 std::atomic<uint32_t> g_stall_polls{0u};  // > 0: the next attention launch is a diagnostic one
 
@@ -1992,8 +1995,8 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
   // only: pairs of CTAs, one work item per pair at a time (see losa_attn_pair.cuh); the single-CTA
   // kernels stay the fallback.  (With 32-key blocks the pair kernel was measured slower than the
   // single-CTA kernel, 6.3 against 5.9 ms for the dense forward at the Wan shape, and is not used.)
-  constexpr bool kPairMode =
-      LOSA_USE_PAIR && D == 128 && R == 128 && C_ >= 64 && (MODE == kDense || MODE == kSparse);
+  constexpr bool kPairMode = LOSA_USE_PAIR && D == 128 && R == 128 && C_ >= 64 &&
+                             (MODE == kDense || MODE == kSparse || (LOSA_PAIR_FUSED && MODE == kFused));
   bool pair = false;  // (a device that cannot hold a pair of these CTAs runs the single-CTA kernel)
   CUtensorMap mkh;
   if constexpr (kPairMode) {
@@ -2120,7 +2123,7 @@ size_t attn_workspace_bytes(AttnMode mode, const Geometry& g, int n_prob) {
   // row: two sets of the halves' row sums, and the rows' weights), per-CTA table of one entry per
   // row and key tile, and the fused step's list of units for the fallback launch
   return kCounterBytes + 5 * kRowstatBytes +
-         (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2) + tl_count_bytes(g, 1);
+         (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2) + 2 * tl_count_bytes(g, 1);
 }
 
 // Batched launch (n_prob > 1, attention-only modes): `layers` is a host array of n_prob problems of

@@ -47,10 +47,12 @@ struct PairControl {
   uint64_t pair_bar[8];    // per (group, lane quarter): the two halves of a row
   uint64_t ref_full[2], ref_empty[2];
   uint64_t item_bar;       // all softmax warps of the CTA, at the end of an item
+  uint64_t fold_bar;       // ... and after the fused step's masses are folded out of the table
   uint64_t drain;
   alignas(16) uint32_t tl[kTlChunks * 32];  // (read in groups of up to four entries with one vector load)
   float ref[2][128];       // the rows' reference, from the group that met the first tile to the other
-  float xch[2][4][128];    // the rows' partial sums at the end of an item (two sets, used in turn)
+  float xch[2][8][128];    // the rows' partial sums at the end of an item (two sets, used in turn):
+                           // four of the rounded weights, four of the unrounded exponentials (fused step)
   uint32_t tmem_base;
   int abort_flag;
   int ovf_unit;
@@ -151,6 +153,7 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   constexpr uint32_t kIdescQK = ptx::idesc_bf16_f32(256, 128, false, false);
   constexpr uint32_t kIdescPV = ptx::idesc_bf16_f32(256, 128, false, true);
   using Ctl = PairControl;
+  constexpr bool kWantMass = (MODE == kFused);  // the construction step: dense O and the block masses
   static_assert(offsetof(PairControl, tl) % 16 == 0, "the tile list is read with 16-byte loads");
 
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -205,6 +208,7 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       ptx::mbar_init(&ctl->ref_empty[i], 8);  // the warps of the other group
     }
     ptx::mbar_init(&ctl->item_bar, 16);
+    ptx::mbar_init(&ctl->fold_bar, 16);
     ptx::mbar_init(&ctl->drain, 2);
     ctl->abort_flag = 0;
     ctl->ovf_unit = -1;
@@ -471,7 +475,13 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     constexpr int kBW = 64 / kHB;                // columns per such block
     uint64_t* const pair_bar = &ctl->pair_bar[grpi * 4 + wl];
     const int quarter = grpi * 2 + half;         // which 32 columns of O this thread writes out
-    uint32_t kq = 0, nod = 0, npair = 0, nitem = 0, nref = 0, te = 0, ent;
+    uint32_t kq = 0, nod = 0, npair = 0, nitem = 0, nref = 0, nfold = 0, te = 0, ent;
+    // fused step: this row's column of the CTA's table of per-block sums of the unrounded
+    // exponentials (one float per row and 64-column half of a key tile when a key block fills the
+    // tile, else one per row and key block)
+    float* const tabf = kWantMass ? reinterpret_cast<float*>(p.table) +
+                                        (int64_t)blockIdx.x * 2 * (int64_t)p.nKb * 256 + row
+                                  : nullptr;
 
     PAIR_TL_NEXT(ent);
     while ((ent >> 28) == 1) {
@@ -484,7 +494,7 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       void* const o_base = (p.problems != nullptr) ? p.problems[pbh / (p.B * p.H)].o : p.o;
       const int T = 2 * pr + (int)rank;
       const int grow = T * 128 + row;
-      float m_ref = 0.f, l = 0.f;
+      float m_ref = 0.f, l = 0.f, le = 0.f;  // le: row sum of the unrounded exponentials (masses, LSE)
       // the reference of the item: set by the group that meets the first key tile this query tile
       // lists, taken over by the other group at its own first such tile (or dropped at the item's end)
       bool item_ref = false, have_ref = false, ref_mine = false, ovf = false;
@@ -595,6 +605,9 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           // The output is normalised by the sum of the weights the tensor core multiplies with V -
           // P as rounded to bf16 - so that o is a weighted mean of V whatever the rounding does.
           float2 racc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+          float2 eacc[kHB];  // fused step: sums of the unrounded exponentials, per block of this half
+#pragma unroll
+          for (int i = 0; i < kHB; ++i) eacc[i] = make_float2(0.f, 0.f);
 #pragma unroll
           for (int c = 0; c < 64; c += 4) {
             if (whole && c == 32) ptx::tmem_wait_ld();
@@ -616,17 +629,30 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             sr[(c >> 1) + 1] = u1;
             ptx::add_bf16x2(racc[0], u0);
             ptx::add_bf16x2(racc[1], u1);
+            if (kWantMass) eacc[c / kBW] = ptx::add2(eacc[c / kBW], ptx::add2(x0, x1));
           }
           const float tsum = (racc[0].x + racc[0].y) + (racc[1].x + racc[1].y);
           ovf = ovf || __any_sync(0xffffffffu, !(tsum <= kSplitSafeSum));
           l += tsum;
           ptx::tmem_st32(tS, &sr[0]);
+          if (kWantMass) {
+#pragma unroll
+            for (int i = 0; i < kHB; ++i) {
+              const float es = eacc[i].x + eacc[i].y;
+              le += es;
+              const int g = (kG >= 2) ? half * kHB + i : 0;
+              const int64_t sb = (kG >= 2) ? (int64_t)(grp[g] & 0xffffu) : (int64_t)(grp[0] & 0xffffu) * 2 + half;
+              if (hv[i] > 0) tabf[sb * 128] = es;
+            }
+          }
         } else {
           // this half of the row lists none of the tile's keys: P = 0
           uint32_t z[32];
 #pragma unroll
           for (int c = 0; c < 32; ++c) z[c] = 0u;
           ptx::tmem_st32(tS, z);
+          // (a key block that fills the tile but ends before this half: its entry of the table is 0)
+          if (kWantMass && kG == 1 && member) tabf[((int64_t)(grp[0] & 0xffffu) * 2 + half) * 128] = 0.f;
         }
         ptx::tmem_wait_st();
         ptx::tc_fence_before_sync();
@@ -650,6 +676,7 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       // the four partial sums of a row (two groups, two halves) meet in shared memory
       float* const xset = &ctl->xch[nitem & 1][0][0];
       xset[quarter * 128 + row] = l;
+      if (kWantMass) xset[(4 + quarter) * 128 + row] = le;
       if (ovf && lane == 0) {
         const int unit = partial ? p.split_first + (w - p.split_first) * p.split_parts + part : w;
         if (atomicExch(&ctl->ovf_unit, unit) != unit) {
@@ -713,6 +740,48 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
           }
         }
+      }
+      if (kWantMass) {
+        // ---- fused construction step: the block masses of this CTA's query tile (Eq. 1).  The
+        // reference did not move during the item, so a row's weight is 1 / (its sum of unrounded
+        // exponentials) and a mass is the mean over the query block's rows of weight x (the row's
+        // sum over the key block).  The table was written by this CTA's softmax threads before the
+        // item's barrier; all 16 warps fold it, key block by key block.
+        if (quarter == 0 && T < p.nQt && grow < p.N && p.lse != nullptr) {
+          const float le_row = (xset[512 + row] + xset[640 + row]) + (xset[768 + row] + xset[896 + row]);
+          p.lse[(int64_t)bh * p.N + grow] = (m_ref + log2f(le_row)) * kLn2;
+        }
+        if (T < p.nQt) {
+          const float* tb = reinterpret_cast<const float*>(p.table) + (int64_t)blockIdx.x * 2 * (int64_t)p.nKb * 256;
+          float iv[4];  // this lane's four rows
+#pragma unroll
+          for (int rr = 0; rr < 4; ++rr) {
+            const int r = rr * 32 + lane;
+            const float le_r = (xset[512 + r] + xset[640 + r]) + (xset[768 + r] + xset[896 + r]);
+            iv[rr] = (T * 128 + r < p.N && le_r > 0.f) ? 1.f / le_r : 0.f;
+          }
+          const int nvalid = min(R, p.N - T * R);
+          for (int u = sw; u < p.nKb; u += 16) {
+            float acc = 0.f;
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr) {
+              const int r = rr * 32 + lane;
+              if (iv[rr] > 0.f) {
+                const float sum = (kG >= 2) ? tb[(int64_t)u * 128 + r]
+                                            : tb[(int64_t)u * 256 + r] + tb[(int64_t)u * 256 + 128 + r];
+                acc += sum * iv[rr];
+              }
+            }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
+            if (lane == 0) p.mass[((int64_t)bh * p.nQb + T) * p.nKb + u] = acc / (float)nvalid;
+          }
+        }
+        // (the table is written again by the next item)
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&ctl->fold_bar);
+        LOSA_WAIT(&ctl->fold_bar, nfold & 1);
+        ++nfold;
       }
     }
   }
