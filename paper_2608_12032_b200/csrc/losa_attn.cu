@@ -33,8 +33,8 @@
 // Every wait is bounded; a wait that expires raises the CTA's abort flag, records
 // LOSA_ERR_TIMEOUT, and all roles leave through the common teardown that frees TMEM.
 //
-// The dense and sparse forward at head dimension 128 with 128-row query blocks and key blocks of 64
-// or 128 keys run in a second kernel, losa_pair_kernel (losa_attn_pair.cuh, included below): pairs
+// The dense and sparse forward and the fused step at head dimension 128 with 128-row query blocks and
+// key blocks of 64 or 128 keys run in a second kernel, losa_pair_kernel (losa_attn_pair.cuh, included below): pairs
 // of CTAs that multiply together (tcgen05.mma.cta_group::2), one query tile and three S buffers per
 // CTA.  This kernel serves every other shape and mode and the fallback launch of all of them.
 #include <cuda.h>

@@ -1,5 +1,6 @@
-// Dense and block-sparse forward (Eq. 4) at head dimension 128 with 128-row query blocks, run by
-// PAIRS of CTAs (clusters of two, one SM each).  Included by losa_attn.cu, inside its namespace.
+// Dense and block-sparse forward (Eq. 4) and the fused construction step (dense forward plus the
+// block masses of Eq. 1) at head dimension 128 with 128-row query blocks, run by PAIRS of CTAs
+// (clusters of two, one SM each).  Included by losa_attn.cu, inside its namespace.
 //
 // A work item is the same pair of consecutive query tiles as in the single-CTA kernel, but each
 // CTA of the pair owns ONE of the two tiles, and the two SMs multiply together: every MMA is a
