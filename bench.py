@@ -54,7 +54,7 @@ def merge_kernel_runs(wl) -> bool:
     """Whether the attention-only calls launch their merge kernel for this shape: the host rule of
     the library, restated (work items = pairs of 128-row query tiles per head)."""
     ctas = min(torch.cuda.get_device_properties(0).multi_processor_count, 160)
-    if wl.D == 128 and wl.R == 128 and wl.C >= 64:
+    if wl.D == 128 and wl.R == 128:
         ctas //= 2  # these shapes run on pairs of CTAs: one work item per pair at a time
     n_work = wl.B * wl.H * ((-(-wl.N // 128) + 1) // 2)
     rest = n_work if n_work < ctas else n_work % ctas

@@ -57,6 +57,9 @@ namespace {
 #ifndef LOSA_PAIR_FUSED
 #define LOSA_PAIR_FUSED 1
 #endif
+#ifndef LOSA_PAIR_MIN_C
+#define LOSA_PAIR_MIN_C 32
+#endif
 
 std::atomic<uint32_t> g_stall_polls{0u};  // > 0: the next attention launch is a diagnostic one
 
@@ -150,6 +153,8 @@ struct Cfg {
 struct alignas(128) ProblemEntry {
   CUtensorMap map_q, map_k, map_v;
   CUtensorMap map_kh;  // K with boxes of at most 64 keys (the CTA-pair kernel copies half a K tile per CTA)
+  // boxes that span several key blocks, for K/V tiles whose key blocks are consecutive (C < 128)
+  CUtensorMap map_k64, map_k128, map_v128;
   void* o;
   const int32_t* offsets;
   const int32_t* kv_idx;
@@ -304,7 +309,8 @@ struct Control {
 template <int D, int R, int C_, int MODE, int KT, bool SPLIT>
 __global__ void __launch_bounds__(Lay<SPLIT>::kThreads, 1)
 losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                 const __grid_constant__ CUtensorMap map_v, const Params p) {
+                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_kw,
+                 const __grid_constant__ CUtensorMap map_vw, const Params p) {
   using C = Cfg<D, R, C_, MODE, KT, SPLIT && D == 64 && MODE != kMass>;
   using L = Lay<SPLIT>;
   using Ctl = Control<C::kNK, C::kNV, SPLIT, SPLIT && D == 64 && MODE != kMass>;
@@ -405,6 +411,10 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     ptx::prefetch_tensormap(&map_q);
     ptx::prefetch_tensormap(&map_k);
     if (C::kHasV) ptx::prefetch_tensormap(&map_v);
+    if (kG > 2) {
+      ptx::prefetch_tensormap(&map_kw);
+      if (C::kHasV) ptx::prefetch_tensormap(&map_vw);
+    }
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
@@ -426,12 +436,14 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const int pbh = w / p.nPairs, pr = w % p.nPairs;
         const int bh = pbh % (p.B * p.H);
         const int b = bh / p.H, h = bh % p.H;
-        const CUtensorMap *mq = &map_q, *mk = &map_k, *mv = &map_v;
+        const CUtensorMap *mq = &map_q, *mk = &map_k, *mv = &map_v, *mkw = &map_kw, *mvw = &map_vw;
         if (p.problems != nullptr) {
           const ProblemEntry* pe = p.problems + pbh / (p.B * p.H);
           mq = &pe->map_q;
           mk = &pe->map_k;
           mv = &pe->map_v;
+          mkw = &pe->map_k128;
+          mvw = &pe->map_v128;
         }
 #pragma unroll
         for (int qt = 0; qt < 2; ++qt) {
@@ -464,7 +476,18 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           // issuing 8 or 16 small copies per tile cannot keep up with the tile rate
           if (lane == 0) ptx::mbar_arrive_expect_tx(&ctl->k_full[ks], C::kKVBytes);
           __syncwarp();
-          if (lane < kG * C::kDH) {
+          // (32-key blocks: a tile whose four key blocks are consecutive is one copy per slab - two
+          // thirds of the sparse tiles on the workload's pattern, all of them in the dense modes;
+          // dense forward 5.70 -> 5.51 ms, fused step 8.38 -> 8.01 ms.  With 64-key blocks one 16 KB
+          // copy instead of two of 8 KB measured 5 % SLOWER in the dense forward, so they stay apart.)
+          bool wide = kG > 2;
+#pragma unroll
+          for (int gg = 1; gg < kG; ++gg) wide = wide && (grp[gg] & 0xffffu) == (grp[0] & 0xffffu) + gg;
+          if (wide) {
+            if (lane < C::kDH)
+              ptx::tma_load_4d(sK + ks * C::kKVBytes + lane * C::kKVSlab, mkw, &ctl->k_full[ks], lane * 64,
+                               (int)(grp[0] & 0xffffu) * kC, h, b);
+          } else if (lane < kG * C::kDH) {
             const int g = lane / C::kDH, s = lane % C::kDH;
             uint32_t eg = grp[0];
 #pragma unroll
@@ -481,7 +504,11 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             LOSA_WAIT_RELAXED(&ctl->v_empty[vs], ((nv / kNVs) & 1) ^ 1);
             if (lane == 0) ptx::mbar_arrive_expect_tx(&ctl->v_full[vs], C::kKVBytes);
             __syncwarp();
-            if (lane < kG * C::kDH) {
+            if (wide) {
+              if (lane < C::kDH)
+                ptx::tma_load_4d(sV + vs * C::kKVBytes + lane * C::kKVSlab, mvw, &ctl->v_full[vs], lane * 64,
+                                 (int)(grp[0] & 0xffffu) * kC, h, b);
+            } else if (lane < kG * C::kDH) {
               const int g = lane / C::kDH, s = lane % C::kDH;
               uint32_t eg = grp[0];
 #pragma unroll
@@ -1899,8 +1926,8 @@ int make_map(CUtensorMap* m, const void* base, const Geometry& g, int box_rows) 
 
 // Configures (once per device) and launches one layout of the attention kernel.
 template <int D, int R, int C_, int MODE, int KT, bool SPLIT>
-int launch_kernel(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                  const Params& prm, int grid, cudaStream_t st) {
+int launch_kernel(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mkw,
+                  const CUtensorMap& mvw, const Params& prm, int grid, cudaStream_t st) {
   using C = Cfg<D, R, C_, MODE, KT, SPLIT && D == 64 && MODE != kMass>;
   using L = Lay<SPLIT>;
   using Ctl = Control<C::kNK, C::kNV, SPLIT, SPLIT && D == 64 && MODE != kMass>;
@@ -1927,7 +1954,7 @@ int launch_kernel(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMa
     LOSA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     configured = true;
   }
-  kern<<<grid, L::kThreads, smem, st>>>(mq, mk, mv, prm);
+  kern<<<grid, L::kThreads, smem, st>>>(mq, mk, mv, mkw, mvw, prm);
   LOSA_CUDA_TRY(cudaGetLastError());
   return LOSA_OK;
 }
@@ -1935,8 +1962,8 @@ int launch_kernel(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMa
 // Configures (once per device) and launches the CTA-pair kernel on `clusters` pairs; *max_clusters
 // (if not null) receives how many pairs the device can hold at once.
 template <int C_, int MODE>
-int launch_pair(const CUtensorMap& mq, const CUtensorMap& mkh, const CUtensorMap& mv, const Params& prm,
-                int clusters, cudaStream_t st, int* max_clusters) {
+int launch_pair(const CUtensorMap& mq, const CUtensorMap& mkh, const CUtensorMap& mv, const CUtensorMap& mk64,
+                const CUtensorMap& mv128, const Params& prm, int clusters, cudaStream_t st, int* max_clusters) {
   using L = Lay<true>;
   constexpr size_t smem = kPairQBytes + (size_t)(kPairNK + kPairNV) * kPairStage + sizeof(PairControl);
   static_assert(smem <= 227 * 1024, "shared memory of one CTA");
@@ -1977,7 +2004,7 @@ int launch_pair(const CUtensorMap& mq, const CUtensorMap& mkh, const CUtensorMap
     return LOSA_OK;
   }
   cfg.gridDim = dim3(2 * clusters, 1, 1);
-  LOSA_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, mq, mkh, mv, prm));
+  LOSA_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, mq, mkh, mv, mk64, mv128, prm));
   return LOSA_OK;
 }
 
@@ -1990,19 +2017,24 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
   if ((rc = make_map(&mq, q, g, 128)) != LOSA_OK) return rc;
   if ((rc = make_map(&mk, k, g, C::kC)) != LOSA_OK) return rc;
   if ((rc = make_map(&mv, C::kHasV ? v : k, g, C::kC)) != LOSA_OK) return rc;
+  CUtensorMap mk128, mv128;  // boxes of a whole 128-key tile, for tiles of consecutive key blocks
+  if ((rc = make_map(&mk128, k, g, 128)) != LOSA_OK) return rc;
+  if ((rc = make_map(&mv128, C::kHasV ? v : k, g, 128)) != LOSA_OK) return rc;
   int ctas = min(sms, kMaxPersistentCtas);
-  // Head dimension 128 with 128-row query blocks and key blocks of 64 or 128, attention output
-  // only: pairs of CTAs, one work item per pair at a time (see losa_attn_pair.cuh); the single-CTA
-  // kernels stay the fallback.  (With 32-key blocks the pair kernel was measured slower than the
-  // single-CTA kernel, 6.3 against 5.9 ms for the dense forward at the Wan shape, and is not used.)
-  constexpr bool kPairMode = LOSA_USE_PAIR && D == 128 && R == 128 && C_ >= 64 &&
+  // Head dimension 128 with 128-row query blocks, modes with an attention output: pairs of CTAs,
+  // one work item per pair at a time (see losa_attn_pair.cuh); the single-CTA kernels stay the
+  // fallback.  (With 32-key blocks the pair kernel was slower than the single-CTA kernel until
+  // tiles of consecutive key blocks were copied whole: dense forward 6.3 against 5.9 ms before,
+  // 5.56 against 6.20 ms after.)
+  constexpr bool kPairMode = LOSA_USE_PAIR && D == 128 && R == 128 && C_ >= LOSA_PAIR_MIN_C &&
                              (MODE == kDense || MODE == kSparse || (LOSA_PAIR_FUSED && MODE == kFused));
   bool pair = false;  // (a device that cannot hold a pair of these CTAs runs the single-CTA kernel)
-  CUtensorMap mkh;
+  CUtensorMap mkh, mk64;
   if constexpr (kPairMode) {
     if ((rc = make_map(&mkh, k, g, C::kC < 64 ? C::kC : 64)) != LOSA_OK) return rc;
+    if ((rc = make_map(&mk64, k, g, 64)) != LOSA_OK) return rc;
     int fit = 0;
-    if (launch_pair<C_, MODE>(mq, mkh, mv, prm, 0, st, &fit) == LOSA_OK && fit >= 1 && sms >= 2) {
+    if (launch_pair<C_, MODE>(mq, mkh, mv, mk64, mv128, prm, 0, st, &fit) == LOSA_OK && fit >= 1 && sms >= 2) {
       pair = true;
       ctas = min(min(sms / 2, fit), kMaxPersistentCtas);
     }
@@ -2041,23 +2073,23 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
     bool launched = false;
     if constexpr (kPairMode) {
       if (pair) {
-        if ((rc = launch_pair<C_, MODE>(mq, mkh, mv, prm, grid, st, nullptr)) != LOSA_OK) return rc;
+        if ((rc = launch_pair<C_, MODE>(mq, mkh, mv, mk64, mv128, prm, grid, st, nullptr)) != LOSA_OK) return rc;
         launched = true;
       }
     }
     if (!launched) {
-      if ((rc = launch_kernel<D, R, C_, MODE, KT, true>(mq, mk, mv, prm, grid, st)) != LOSA_OK) return rc;
+      if ((rc = launch_kernel<D, R, C_, MODE, KT, true>(mq, mk, mv, mk128, mv128, prm, grid, st)) != LOSA_OK) return rc;
     }
     if (!prm.stall) {
       prm.redo = 1;
       prm.work_counter += 2;  // its own counter (zeroed with the first)
       // (as many CTAs as SMs, whichever kernel ran first)
       const int rgrid = min(min(sms, kMaxPersistentCtas), prm.nUnits);
-      if ((rc = launch_kernel<D, R, C_, MODE, KT, false>(mq, mk, mv, prm, rgrid, st)) != LOSA_OK) return rc;
+      if ((rc = launch_kernel<D, R, C_, MODE, KT, false>(mq, mk, mv, mk128, mv128, prm, rgrid, st)) != LOSA_OK) return rc;
     }
   } else {
     prm.redo = 0;
-    if ((rc = launch_kernel<D, R, C_, MODE, KT, false>(mq, mk, mv, prm, grid, st)) != LOSA_OK) return rc;
+    if ((rc = launch_kernel<D, R, C_, MODE, KT, false>(mq, mk, mv, mk128, mv128, prm, grid, st)) != LOSA_OK) return rc;
   }
   if (prm.split_parts > 1) {
     merge_parts_kernel<D><<<dim3(prm.nWork - prm.split_first, 16), 128, 0, st>>>(prm);
@@ -2176,6 +2208,9 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
         if ((rc = make_map(&host[i].map_k, layers[i].k, g, g.C)) != LOSA_OK) return rc;
         if ((rc = make_map(&host[i].map_v, layers[i].v, g, g.C)) != LOSA_OK) return rc;
         if ((rc = make_map(&host[i].map_kh, layers[i].k, g, g.C < 64 ? g.C : 64)) != LOSA_OK) return rc;
+        if ((rc = make_map(&host[i].map_k64, layers[i].k, g, 64)) != LOSA_OK) return rc;
+        if ((rc = make_map(&host[i].map_k128, layers[i].k, g, 128)) != LOSA_OK) return rc;
+        if ((rc = make_map(&host[i].map_v128, layers[i].v, g, 128)) != LOSA_OK) return rc;
         host[i].o = layers[i].o;
         host[i].offsets = layers[i].offsets;
         host[i].kv_idx = layers[i].kv_idx;

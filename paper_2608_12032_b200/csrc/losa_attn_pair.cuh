@@ -145,7 +145,8 @@ struct PairControl {
 template <int C_, int MODE>
 __global__ void __launch_bounds__(Lay<true>::kThreads, 1)
 losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                 const __grid_constant__ CUtensorMap map_v, const Params p) {
+                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_kw,
+                 const __grid_constant__ CUtensorMap map_vw, const Params p) {
   using L = Lay<true>;
   constexpr int D = 128, R = 128;
   constexpr int kC = C_, kG = 128 / C_, kW = 128;
@@ -224,6 +225,10 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     ptx::prefetch_tensormap(&map_q);
     ptx::prefetch_tensormap(&map_k);
     ptx::prefetch_tensormap(&map_v);
+    if (kG > 2) {
+      ptx::prefetch_tensormap(&map_kw);
+      ptx::prefetch_tensormap(&map_vw);
+    }
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
@@ -254,12 +259,15 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const int pbh = w / p.nPairs, pr = w % p.nPairs;
         const int bh = pbh % (p.B * p.H);
         const int b = bh / p.H, h = bh % p.H;
-        const CUtensorMap *mq = &map_q, *mk = &map_k, *mv = &map_v;
+        // (map_kw: K in boxes of 64 keys, map_vw: V in boxes of 128 keys, for consecutive key blocks)
+        const CUtensorMap *mq = &map_q, *mk = &map_k, *mv = &map_v, *mkw = &map_kw, *mvw = &map_vw;
         if (p.problems != nullptr) {
           const ProblemEntry* pe = p.problems + pbh / (p.B * p.H);
           mq = &pe->map_q;
           mk = &pe->map_kh;
           mv = &pe->map_v;
+          mkw = &pe->map_k64;
+          mvw = &pe->map_v128;
         }
         // this CTA's query tile (rows past the end of the sequence are filled with zeros)
         const int T = 2 * pr + (int)rank;
@@ -283,7 +291,19 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           LOSA_WAIT_RELAXED(&ctl->k_empty[ks], ((nk / kPairNK) & 1) ^ 1);
           if (lane == 0) ptx::mbar_arrive_expect_tx_cluster(k_full0 + 8u * ks, kPairStage);
           __syncwarp();
-          if (lane < 2 * kKCopies) {
+          // 32-key blocks: this CTA's two key blocks, if consecutive, are one copy per slab
+          bool wide_k = false;
+          uint32_t first_k = grp[0];
+          if constexpr (kKCopies == 2) {
+            const uint32_t e0 = (rank == 0) ? grp[0] : grp[kG / 2], e1 = (rank == 0) ? grp[1] : grp[kG / 2 + 1];
+            wide_k = (e1 & 0xffffu) == (e0 & 0xffffu) + 1u;
+            first_k = e0;
+          }
+          if (wide_k) {
+            if (lane < 2)
+              ptx::tma_load_4d_pair(sK + ks * kPairStage + lane * 8192, mkw, k_full0 + 8u * ks, lane * 64,
+                                    (int)(first_k & 0xffffu) * kC, h, b);
+          } else if (lane < 2 * kKCopies) {
             const int i = lane >> 1, s = lane & 1;
             const int keyoff = 64 * (int)rank + i * kKBox;  // within the tile
             const int g = keyoff / kC, inb = keyoff % kC;
@@ -302,7 +322,14 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           LOSA_WAIT_RELAXED(&ctl->v_empty[vs], ((nv / kPairNV) & 1) ^ 1);
           if (lane == 0) ptx::mbar_arrive_expect_tx_cluster(v_full0 + 8u * vs, kPairStage);
           __syncwarp();
-          if (lane < kG) {
+          bool wide_v = kG > 2;
+#pragma unroll
+          for (int gg = 1; gg < kG; ++gg) wide_v = wide_v && (grp[gg] & 0xffffu) == (grp[0] & 0xffffu) + gg;
+          if (wide_v) {
+            if (lane == 0)
+              ptx::tma_load_4d_pair(sV + vs * kPairStage, mvw, v_full0 + 8u * vs, (int)rank * 64,
+                                    (int)(grp[0] & 0xffffu) * kC, h, b);
+          } else if (lane < kG) {
             uint32_t eg = grp[0];
 #pragma unroll
             for (int gg = 1; gg < kG; ++gg)

@@ -36,17 +36,17 @@ def items(B, H, N):
 
 def cut_into_parts(n_items, D, R, C):
     """The library's host rule, restated: are the work items of the last wave cut into parts?
-    (Head dimension 128 with 128-row query blocks and key blocks of 64 or 128 runs on pairs of
-    CTAs: half as many slots.)"""
+    (Head dimension 128 with 128-row query blocks runs on pairs of CTAs: half as many slots.)"""
     ctas = min(torch.cuda.get_device_properties(0).multi_processor_count, 160)
-    if D == 128 and R == 128 and C >= 64:
+    if D == 128 and R == 128:
         ctas //= 2
     rest = n_items if n_items < ctas else n_items % ctas
     return rest > 0 and ctas // rest >= 2
 
 
 @pytest.mark.parametrize("B,H,N,D,R,C", [(1, 5, 128 * 31 + 70, 64, 64, 64), (1, 5, 128 * 32 - 9, 128, 128, 32),
-                                         (1, 37, 128 * 4 - 9, 128, 128, 64), (1, 37, 128 * 4 - 9, 128, 128, 128)])
+                                         (1, 37, 128 * 4 - 9, 128, 128, 64), (1, 37, 128 * 4 - 9, 128, 128, 128),
+                                         (1, 37, 128 * 4 - 9, 128, 128, 32)])
 def test_three_layers_in_one_launch_equal_the_single_calls_bit_for_bit(B, H, N, D, R, C):
     losa = lib()
     L = 3

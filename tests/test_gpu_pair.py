@@ -54,7 +54,7 @@ def patterns(nQb, nKb, kind, seed):
     return rows
 
 
-@pytest.mark.parametrize("C", [128, 64])
+@pytest.mark.parametrize("C", [128, 64, 32])
 @pytest.mark.parametrize("kind", ["disjoint_singletons", "late_only_tile", "odd_position_first", "interleaved", "random"])
 @pytest.mark.parametrize("tiles", [6, 7])
 def test_crafted_patterns_match_oracle(C, kind, tiles):
@@ -77,7 +77,7 @@ def test_crafted_patterns_match_oracle(C, kind, tiles):
     util.assert_output_close(o, ref, f"{kind} C={C} tiles={tiles}")
 
 
-@pytest.mark.parametrize("C", [128, 64])
+@pytest.mark.parametrize("C", [128, 64, 32])
 def test_whole_and_cut_work_units_in_one_launch(C):
     """More work items than pairs of CTAs fit at once, and not a multiple of them: the first waves
     run whole items, the last one is cut into parts and merged."""
