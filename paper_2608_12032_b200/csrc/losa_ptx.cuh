@@ -360,7 +360,7 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
   return ok != 0;
 }
 
-// mbar_wait / mbar_wait_relaxed for a barrier that the other CTA of the pair arrives on
+// mbar_wait for a barrier whose data another CTA of the pair wrote through shared memory
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                                   uint32_t limit) {
   for (uint32_t it = 0; it < limit; ++it) {
@@ -368,18 +368,6 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
     if (it >= kFastPolls) {
       if (*abort_flag) return false;
       __nanosleep(256);
-    }
-  }
-  return false;
-}
-
-__device__ __forceinline__ bool mbar_wait_cluster_relaxed(uint64_t* bar, uint32_t parity,
-                                                          volatile int* abort_flag, uint32_t limit) {
-  for (uint32_t it = 0; it < limit; ++it) {
-    if (mbar_try_wait_cluster(bar, parity)) return true;
-    if (it >= 4) {
-      if ((it & 1023u) == 0 && *abort_flag) return false;
-      __nanosleep(it < 64 ? 64 : 256);
     }
   }
   return false;
