@@ -64,8 +64,10 @@ enum {
   LOSA_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed                            */
   LOSA_ERR_TIMEOUT = -6,     /* a bounded device-side wait expired (device-side)             */
   LOSA_ERR_BAD_INDEX = -7,   /* kv_idx / offsets out of range or not ascending (device-side) */
-  LOSA_ERR_BAD_MASS = -8     /* losa_select saw a negative, NaN or > 8 mass, or a row whose
+  LOSA_ERR_BAD_MASS = -8,    /* losa_select saw a negative, NaN or > 8 mass, or a row whose
                                 masses add up to more than 8 (device-side)                   */
+  LOSA_ERR_INTERNAL = -9     /* checked build only (-DLOSA_CHECKED=1): a kernel computed an index
+                                outside its buffer; the access was skipped (device-side)     */
 };
 
 enum {

@@ -14,7 +14,8 @@ from typing import Optional, Tuple
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "liblosa.so")
+# (LOSA_LIBRARY selects another build of the same library, e.g. the checked build of the kernels)
+LIB_PATH = os.environ.get("LOSA_LIBRARY") or os.path.join(_PKG, "liblosa.so")
 
 LOSA_OP_BLOCK_MASS, LOSA_OP_SELECT, LOSA_OP_SPARSE_ATTN, LOSA_OP_ATTN, LOSA_OP_ATTN_MASS = 0, 1, 2, 3, 4
 LOSA_DTYPE_BF16, LOSA_DTYPE_F32 = 0, 1

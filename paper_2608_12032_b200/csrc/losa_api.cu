@@ -323,6 +323,7 @@ const char* losa_status_string(int status) {
     case LOSA_ERR_TIMEOUT: return "LOSA_ERR_TIMEOUT";
     case LOSA_ERR_BAD_INDEX: return "LOSA_ERR_BAD_INDEX";
     case LOSA_ERR_BAD_MASS: return "LOSA_ERR_BAD_MASS";
+    case LOSA_ERR_INTERNAL: return "LOSA_ERR_INTERNAL";
   }
   return "LOSA_ERR_UNKNOWN";
 }

@@ -196,6 +196,8 @@ struct Params {
   int* redo_count;
   int* redo_list;
   int redo;             // this launch processes redo_list[0 .. *redo_count) instead of all units
+  // extents of the buffers the kernels index into (elements), for the checked build
+  long long cap_part_rows, cap_table_floats, cap_mass, cap_lse, cap_units;
   uint32_t wait_polls;  // bound of every device-side wait, in polls (ptx::kWaitPolls)
   int stall;            // diagnostic launch: the scheduler publishes nothing, so that every wait runs out
 };
@@ -228,6 +230,20 @@ struct Control {
   uint64_t rot_s_full[ROT ? 6 : 1], rot_p_ready[ROT ? 6 : 1];
   uint64_t pv_done[ROT ? 3 : 1];  // per buffer: the product that read its P has run
 };
+
+// Checked build (-DLOSA_CHECKED=1, a substitute for a memory checker): every index the kernels
+// compute into the workspace, the masses or the log-sum-exp is compared with the extent of its
+// buffer; one that falls outside is recorded as LOSA_ERR_INTERNAL and the access is skipped (or
+// redirected to element 0 of the same buffer).  The ordinary build compiles the checks away.
+#ifndef LOSA_CHECKED
+#define LOSA_CHECKED 0
+#endif
+#if LOSA_CHECKED
+#define LOSA_IN_RANGE(idx, extent) \
+  (((unsigned long long)(idx) < (unsigned long long)(extent)) || (report_error(p.status, LOSA_ERR_INTERNAL), false))
+#else
+#define LOSA_IN_RANGE(idx, extent) true
+#endif
 
 #define LOSA_WAIT_RELAXED(bar, parity)                                   \
   do {                                                                   \
@@ -871,7 +887,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // the unit's merged tile list was built before the launch: stream it into the ring,
         // 32 entries per step, so that this warp takes next to no issue slots from the softmax
         // warps of its scheduler partition
-        const int cnt = __ldg(p.tl_count + unit);
+        const int cnt = LOSA_IN_RANGE(unit, p.cap_units) ? min(__ldg(p.tl_count + unit), p.tl_cap) : 0;
         const uint32_t* src = p.tl_entries + (int64_t)unit * p.tl_cap;
         for (int base = 0; base < cnt; base += 32) {
           const int n = min(32, cnt - base);
@@ -1160,7 +1176,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const int64_t off = (int64_t)b * p.sb + (int64_t)h * p.sh + (int64_t)grow * p.sn;
           const int64_t pslot =
               ((((int64_t)(w - p.split_first) * p.split_parts + part) * 2 + qt) * 128 + row);
-          if (partial) p.part_ml[pslot] = make_float2(m_ref, l);
+          if (partial && LOSA_IN_RANGE(pslot, p.cap_part_rows)) p.part_ml[pslot] = make_float2(m_ref, l);
           if (pv_item > 0) {
             // o_done advances once per item, so its parity is unambiguous here (a product's own barrier may be
             // one, two or three phases from this warp's last look at it)
@@ -1180,7 +1196,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
             if (partial) {
               // a part of the key range: unnormalised O, merged with the other parts afterwards
-              float4* dst = reinterpret_cast<float4*>(p.part_o + pslot * D + c0);
+              float4* dst = reinterpret_cast<float4*>(p.part_o + (LOSA_IN_RANGE(pslot, p.cap_part_rows) ? pslot : 0) * D + c0);
 #pragma unroll
               for (int c = 0; c < 32; c += 4)
                 dst[c >> 2] = make_float4(__uint_as_float(r[c]), __uint_as_float(r[c + 1]),
@@ -1220,7 +1236,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (T < p.nQt) {
           const bool valid = grow < p.N;
           rs[row] = make_float2(m_ref, (valid && l > 0.f) ? 1.f / l : 0.f);
-          if (p.lse != nullptr && valid)
+          if (p.lse != nullptr && valid && LOSA_IN_RANGE((int64_t)bh * p.N + grow, p.cap_lse))
             p.lse[(int64_t)bh * p.N + grow] = (m_ref + log2f(l)) * kLn2;
         }
         ptx::mbar_arrive(&ctl->wg_bar[qt]);  // warpgroup sync with a bounded wait
@@ -1252,7 +1268,10 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               const int g = T * kQBT + q;
               if (lane == 0 && g < p.nQb) {
                 const int nvalid = min(R, p.N - g * R);
-                p.mass[((int64_t)bh * p.nQb + g) * p.nKb + u] = a / (float)nvalid;
+                {
+                  const int64_t mi = ((int64_t)bh * p.nQb + g) * p.nKb + u;
+                  if (LOSA_IN_RANGE(mi, p.cap_mass)) p.mass[mi] = a / (float)nvalid;
+                }
               }
             }
           }
@@ -1476,7 +1495,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               le += es;
               const int g = (kG >= 2) ? half * kHB + i : 0;
               const int64_t sb = (kG >= 2) ? (int64_t)(grp[g] & 0xffffu) : (int64_t)(grp[0] & 0xffffu) * 2 + half;
-              if (hv[i] > 0) tabf[sb * 128] = es;
+              if (hv[i] > 0 && LOSA_IN_RANGE(sb * 128 + row, p.cap_table_floats)) tabf[sb * 128] = es;
             }
           }
         } else {
@@ -1493,7 +1512,9 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             if (lane == 0) ptx::mbar_arrive(&ctl->s_free[qt][nsub % kNS]);
           }
           // (a key block that fills the tile but ends before this half: its entry of the table is 0)
-          if (C::kWantMass && kG == 1 && pair_mine) tabf[((int64_t)(grp[0] & 0xffffu) * 2 + half) * 128] = 0.f;
+          if (C::kWantMass && kG == 1 && pair_mine &&
+              LOSA_IN_RANGE(((int64_t)(grp[0] & 0xffffu) * 2 + half) * 128 + row, p.cap_table_floats))
+            tabf[((int64_t)(grp[0] & 0xffffu) * 2 + half) * 128] = 0.f;
         }
         if (C::kHasV) {
           ptx::tmem_wait_st();
@@ -1538,7 +1559,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const int64_t off = (int64_t)b * p.sb + (int64_t)h * p.sh + (int64_t)grow * p.sn;
         const int64_t pslot =
             ((((int64_t)(w - p.split_first) * p.split_parts + part) * 2 + qt) * 128 + row);
-        if (partial) p.part_ml[pslot] = make_float2(m_ref, l);
+        if (partial && LOSA_IN_RANGE(pslot, p.cap_part_rows)) p.part_ml[pslot] = make_float2(m_ref, l);
         if (pv_item > 0) {
           LOSA_WAIT(&ctl->o_done[qt], nod & 1);
           ++nod;
@@ -1555,7 +1576,7 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             for (int c = 0; c < 32; ++c) r[c] = 0u;
           }
           if (partial) {
-            float4* dst = reinterpret_cast<float4*>(p.part_o + pslot * D + c0);
+            float4* dst = reinterpret_cast<float4*>(p.part_o + (LOSA_IN_RANGE(pslot, p.cap_part_rows) ? pslot : 0) * D + c0);
 #pragma unroll
             for (int c = 0; c < 32; c += 4)
               dst[c >> 2] = make_float4(__uint_as_float(r[c]), __uint_as_float(r[c + 1]),
@@ -1595,7 +1616,8 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (half == 0 && T < p.nQt) {
           const bool valid = grow < p.N;
           inv_rows[row] = (valid && le > 0.f) ? 1.f / le : 0.f;
-          if (p.lse != nullptr && valid) p.lse[(int64_t)bh * p.N + grow] = (m_ref + log2f(le)) * kLn2;
+          if (p.lse != nullptr && valid && LOSA_IN_RANGE((int64_t)bh * p.N + grow, p.cap_lse))
+            p.lse[(int64_t)bh * p.N + grow] = (m_ref + log2f(le)) * kLn2;
         }
         ptx::mbar_arrive(&ctl->wg_bar[qt]);  // all eight warps of the query tile, with a bounded wait
         LOSA_WAIT(&ctl->wg_bar[qt], nwg & 1);
@@ -1629,7 +1651,10 @@ losa_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               const int g = T * kQBT + q;
               if (lane == 0 && g < p.nQb) {
                 const int nvalid = min(R, p.N - g * R);
-                p.mass[((int64_t)bh * p.nQb + g) * p.nKb + u] = a2 / (float)nvalid;
+                {
+                  const int64_t mi = ((int64_t)bh * p.nQb + g) * p.nKb + u;
+                  if (LOSA_IN_RANGE(mi, p.cap_mass)) p.mass[mi] = a2 / (float)nvalid;
+                }
               }
             }
           }
@@ -2232,6 +2257,11 @@ int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, 
       prm.redo_list = reinterpret_cast<int*>(reinterpret_cast<char*>(prm.table) +
                                              (size_t)kMaxPersistentCtas * 2 * (size_t)g.nKb * 128 * sizeof(float2));
   }
+  prm.cap_part_rows = (long long)kMaxPersistentCtas * 2 * 128;
+  prm.cap_table_floats = (long long)g.nKb * 256;
+  prm.cap_mass = (long long)g.B * g.H * g.nQb * g.nKb;
+  prm.cap_lse = (long long)g.B * g.H * g.N;
+  prm.cap_units = (long long)max_units(g, n_prob);
   prm.scale_log2 = g.scale * kLog2e;
   int rc = LOSA_OK;
   const DeviceState* dev = device_state(&rc);

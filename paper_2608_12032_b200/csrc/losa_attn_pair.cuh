@@ -442,7 +442,7 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const int pr = w % p.nPairs;
         PAIR_TL_PUT(kTlItem | flags | (uint32_t)w);
         if (MODE == kSparse) {
-          const int cnt = __ldg(p.tl_count + unit);
+          const int cnt = LOSA_IN_RANGE(unit, p.cap_units) ? min(__ldg(p.tl_count + unit), p.tl_cap) : 0;
           const uint32_t* src = p.tl_entries + (int64_t)unit * p.tl_cap;
           for (int base = 0; base < cnt; base += 32) {
             const int n = min(32, cnt - base);
@@ -651,7 +651,7 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               le += es;
               const int g = (kG >= 2) ? half * kHB + i : 0;
               const int64_t sb = (kG >= 2) ? (int64_t)(grp[g] & 0xffffu) : (int64_t)(grp[0] & 0xffffu) * 2 + half;
-              if (hv[i] > 0) tabf[sb * 128] = es;
+              if (hv[i] > 0 && LOSA_IN_RANGE(sb * 128 + row, p.cap_table_floats)) tabf[sb * 128] = es;
             }
           }
         } else {
@@ -661,7 +661,9 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           for (int c = 0; c < 32; ++c) z[c] = 0u;
           ptx::tmem_st32(tS, z);
           // (a key block that fills the tile but ends before this half: its entry of the table is 0)
-          if (kWantMass && kG == 1 && member) tabf[((int64_t)(grp[0] & 0xffffu) * 2 + half) * 128] = 0.f;
+          if (kWantMass && kG == 1 && member &&
+              LOSA_IN_RANGE(((int64_t)(grp[0] & 0xffffu) * 2 + half) * 128 + row, p.cap_table_floats))
+            tabf[((int64_t)(grp[0] & 0xffffu) * 2 + half) * 128] = 0.f;
         }
         ptx::tmem_wait_st();
         ptx::tc_fence_before_sync();
@@ -704,7 +706,7 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const float inv = (l > 0.f) ? 1.f / l : 0.f;
         const int64_t off = (int64_t)b * p.sb + (int64_t)h * p.sh + (int64_t)grow * p.sn;
         const int64_t pslot = ((((int64_t)(w - p.split_first) * p.split_parts + part) * 2 + (int)rank) * 128 + row);
-        if (partial && quarter == 0 && T < p.nQt) p.part_ml[pslot] = make_float2(m_ref, l);
+        if (partial && quarter == 0 && T < p.nQt && LOSA_IN_RANGE(pslot, p.cap_part_rows)) p.part_ml[pslot] = make_float2(m_ref, l);
         const int c0 = quarter * 32;
         uint32_t r[32];
         if (pv_item > 0) {
@@ -723,7 +725,7 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         if (partial) {
           if (T < p.nQt) {
-            float4* dst = reinterpret_cast<float4*>(p.part_o + pslot * D + c0);
+            float4* dst = reinterpret_cast<float4*>(p.part_o + (LOSA_IN_RANGE(pslot, p.cap_part_rows) ? pslot : 0) * D + c0);
 #pragma unroll
             for (int c = 0; c < 32; c += 4)
               dst[c >> 2] = make_float4(__uint_as_float(r[c]), __uint_as_float(r[c + 1]),
@@ -756,7 +758,8 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // exponentials) and a mass is the mean over the query block's rows of weight x (the row's
         // sum over the key block).  The table was written by this CTA's softmax threads before the
         // item's barrier; all 16 warps fold it, key block by key block.
-        if (quarter == 0 && T < p.nQt && grow < p.N && p.lse != nullptr) {
+        if (quarter == 0 && T < p.nQt && grow < p.N && p.lse != nullptr &&
+            LOSA_IN_RANGE((int64_t)bh * p.N + grow, p.cap_lse)) {
           const float le_row = (xset[512 + row] + xset[640 + row]) + (xset[768 + row] + xset[896 + row]);
           p.lse[(int64_t)bh * p.N + grow] = (m_ref + log2f(le_row)) * kLn2;
         }
@@ -783,7 +786,8 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
-            if (lane == 0) p.mass[((int64_t)bh * p.nQb + T) * p.nKb + u] = acc / (float)nvalid;
+            const int64_t mi = ((int64_t)bh * p.nQb + T) * p.nKb + u;
+            if (lane == 0 && LOSA_IN_RANGE(mi, p.cap_mass)) p.mass[mi] = acc / (float)nvalid;
           }
         }
         // (the table is written again by the next item)
