@@ -117,3 +117,36 @@ def test_same_call_twice_gives_the_same_bits():
         again = losa.losa_sparse_attn(q, k, v, offd, idxd, R, C, out_dtype=torch.float32)
         assert torch.equal(first, again)
     assert losa.losa_async_status() == 0
+
+
+@pytest.mark.parametrize("Dh,Rq,Ck", [(128, 128, 128), (64, 64, 64)])
+def test_two_streams_with_their_own_workspaces_do_not_disturb_each_other(Dh, Rq, Ck):
+    """Calls on different streams may overlap on the GPU when each has its own workspace and output
+    (the header's rule): persistent kernels of two launches then share the SMs.  Each stream's results
+    must equal, bit for bit, what the same calls give alone."""
+    losa = lib()
+    B, H, N = 1, 6, 128 * 11 + 40
+    nQb, nKb = -(-N // Rq), -(-N // Ck)
+    data = []
+    for i in range(2):
+        q, k, v = (util.rand_bf16((B, H, N, Dh), 1200 + 10 * i + j, 1.5).cuda() for j in range(3))
+        off, idx = util.random_csr(B * H * nQb, nKb, 40 + i, 0.5)
+        data.append((q, k, v, torch.from_numpy(off).cuda(), torch.from_numpy(idx).cuda()))
+    alone = []
+    for q, k, v, off, idx in data:
+        alone.append((losa.losa_sparse_attn(q, k, v, off, idx, Rq, Ck, out_dtype=torch.float32),
+                      losa.losa_attn(q, k, v, Rq, Ck, out_dtype=torch.float32)))
+    torch.cuda.synchronize()
+    assert losa.losa_async_status() == 0
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    results = [[], []]
+    for rep in range(4):
+        for i, (q, k, v, off, idx) in enumerate(data):
+            with torch.cuda.stream(streams[i]):
+                results[i].append((losa.losa_sparse_attn(q, k, v, off, idx, Rq, Ck, out_dtype=torch.float32),
+                                   losa.losa_attn(q, k, v, Rq, Ck, out_dtype=torch.float32)))
+    torch.cuda.synchronize()
+    assert losa.losa_async_status() == 0
+    for i in range(2):
+        for o_s, o_d in results[i]:
+            assert torch.equal(o_s, alone[i][0]) and torch.equal(o_d, alone[i][1])
