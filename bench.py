@@ -51,11 +51,12 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 
 def merge_kernel_runs(wl) -> bool:
-    """Whether the attention-only calls launch their merge kernel for this shape: the host rule of
-    the library, restated (work items = pairs of 128-row query tiles per head)."""
-    ctas = min(torch.cuda.get_device_properties(0).multi_processor_count, 160)
-    if wl.D == 128 and wl.R == 128:
-        ctas //= 2  # these shapes run on pairs of CTAs: one work item per pair at a time
+    """Whether the attention-only calls launch their merge kernel for this shape: the library says how
+    many work slots a call occupies; work items are pairs of 128-row query tiles per head, and the
+    items of a last, partly filled wave are cut into parts (at most 8, at most one per key block)."""
+    from paper_2608_12032_b200 import binding
+    prob = binding.Problem(wl.B, wl.H, wl.N, wl.D, wl.R, wl.C, wl.H * wl.N * wl.D, wl.N * wl.D, wl.D, 0.0)
+    ctas = binding.losa_work_slots(binding.LOSA_OP_SPARSE_ATTN, prob)
     n_work = wl.B * wl.H * ((-(-wl.N // 128) + 1) // 2)
     rest = n_work if n_work < ctas else n_work % ctas
     parts = min(ctas // rest, 8, -(-wl.N // wl.C)) if rest else 1

@@ -234,6 +234,15 @@ int losa_sparse_attn_batched(const losa_problem_t* p, int32_t n_layers, const lo
 /* Workspace of a batched call (op: LOSA_OP_SPARSE_ATTN); 0 for an invalid problem or count. */
 size_t losa_workspace_bytes_batched(int op, const losa_problem_t* p, int32_t n_layers);
 
+/* How many work slots (persistent CTAs, or pairs of CTAs where the kernel pairs them) a call
+ * of kind `op` (a LOSA_OP_* attention call) occupies on the current device.  A call's work items -
+ * pairs of 128-row query tiles per (batch, head) - are spread over these slots, and the items of
+ * a last, partly filled wave are cut into parts and merged; callers that compare results bit for
+ * bit across calls of different sizes need this number.  0 for an invalid problem or op.
+ * (On a device that cannot hold a pair of CTAs the paired kernels fall back to single CTAs; the
+ * number returned does not know that.) */
+int32_t losa_work_slots(int op, const losa_problem_t* p);
+
 /* Dense softmax attention o = softmax(q k^T * scale) v over the N valid keys: the paper's
  * dense steps up to the construction step, and this library's own dense baseline.
  * Same tensors and workspace rule as losa_sparse_attn, without the CSR. */

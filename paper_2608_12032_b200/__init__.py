@@ -19,6 +19,7 @@ from .binding import (  # noqa: F401
     losa_sparse_attn_batched,
     losa_status_string,
     losa_validate_csr,
+    losa_work_slots,
     losa_workspace_bytes,
     losa_workspace_bytes_batched,
     make_problem,

@@ -25,6 +25,7 @@ EXPORTS = (
     "losa_attn_mass", "losa_select_topk", "losa_row_recall",
     "losa_select_noalloc", "losa_validate_csr", "losa_async_status", "losa_status_string", "losa_last_cuda_error",
     "losa_debug_stall_next_launch", "losa_sparse_attn_batched", "losa_workspace_bytes_batched",
+    "losa_work_slots",
 )
 
 
@@ -85,6 +86,8 @@ def _lib():
         lib.losa_sparse_attn_batched.argtypes = [pp, i32, ctypes.POINTER(Layer), ctypes.c_int, vp, sz, vp]
         lib.losa_workspace_bytes_batched.restype = sz
         lib.losa_workspace_bytes_batched.argtypes = [ctypes.c_int, pp, i32]
+        lib.losa_work_slots.restype = i32
+        lib.losa_work_slots.argtypes = [ctypes.c_int, pp]
         lib.losa_attn.restype = ctypes.c_int
         lib.losa_attn.argtypes = [pp, vp, vp, vp, vp, ctypes.c_int, vp, sz, vp]
         lib.losa_attn_mass.restype = ctypes.c_int
@@ -134,6 +137,11 @@ def _same_layout(ref: torch.Tensor, *others: torch.Tensor) -> None:
 
 def losa_workspace_bytes(op: int, problem: Problem) -> int:
     return int(_lib().losa_workspace_bytes(op, ctypes.byref(problem)))
+
+
+def losa_work_slots(op: int, problem: Problem) -> int:
+    """Work slots (persistent CTAs, or pairs of them) an attention call of this kind occupies."""
+    return int(_lib().losa_work_slots(op, ctypes.byref(problem)))
 
 
 def _workspace(op: int, problem: Problem, device, ws: Optional[torch.Tensor]) -> Tuple[Optional[torch.Tensor], int]:

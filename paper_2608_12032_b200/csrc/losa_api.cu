@@ -130,6 +130,21 @@ size_t losa_workspace_bytes(int op, const losa_problem_t* p) {
   return 0;
 }
 
+int32_t losa_work_slots(int op, const losa_problem_t* p) {
+  Geometry g;
+  if (!p || make_geometry(p, &g) != LOSA_OK) return 0;
+  int rc = LOSA_OK;
+  const DeviceState* dev = device_state(&rc);
+  if (!dev) return 0;
+  switch (op) {
+    case LOSA_OP_BLOCK_MASS: return attn_work_slots(kMass, g, dev->sm_count);
+    case LOSA_OP_SPARSE_ATTN: return attn_work_slots(kSparse, g, dev->sm_count);
+    case LOSA_OP_ATTN: return attn_work_slots(kDense, g, dev->sm_count);
+    case LOSA_OP_ATTN_MASS: return attn_work_slots(kFused, g, dev->sm_count);
+  }
+  return 0;
+}
+
 int losa_block_mass(const losa_problem_t* p, const void* q, const void* k, float* mass, float* lse,
                     void* ws, size_t ws_bytes, void* cuda_stream) {
   Geometry g;

@@ -2163,6 +2163,16 @@ size_t tl_entries_bytes(const Geometry& g, int n_prob) {
 
 void arm_stalled_launch(uint32_t polls) { g_stall_polls.store(polls); }
 
+// Work slots (persistent CTAs, or pairs of CTAs) that a call of this kind occupies on a device
+// with `sms` multiprocessors: the host rule of launch_t, for callers that want to know how the
+// work items are spread (which of them the last wave cuts into parts).
+int attn_work_slots(AttnMode mode, const Geometry& g, int sms) {
+  const int ctas = sms < kMaxPersistentCtas ? sms : kMaxPersistentCtas;
+  const bool pair = LOSA_USE_PAIR && g.D == 128 && g.R == 128 && g.C >= LOSA_PAIR_MIN_C &&
+                    (mode == kDense || mode == kSparse || (LOSA_PAIR_FUSED && mode == kFused)) && sms >= 2;
+  return pair ? ctas / 2 : ctas;
+}
+
 size_t attn_workspace_bytes(AttnMode mode, const Geometry& g, int n_prob) {
   // attention output: counter, then one slot per partial unit (at most one per CTA) holding the
   // rows' (max, sum) and unnormalised O of both query tiles

@@ -76,6 +76,7 @@ enum AttnMode { kDense = 0, kSparse = 1, kMass = 2, kFused = 3 };  // kFused: de
 
 size_t attn_workspace_bytes(AttnMode mode, const Geometry& g, int n_prob = 1);
 void arm_stalled_launch(uint32_t polls);  // the next attention launch publishes no work (diagnostic)
+int attn_work_slots(AttnMode mode, const Geometry& g, int sms);
 int launch_attn(AttnMode mode, const Geometry& g, const void* q, const void* k, const void* v,
                 const int32_t* offsets, const int32_t* kv_idx, void* o, int o_dtype, float* mass,
                 float* lse, void* ws, cudaStream_t st, int n_prob = 1,

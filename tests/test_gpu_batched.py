@@ -34,12 +34,12 @@ def items(B, H, N):
     return B * H * ((-(-N // 128) + 1) // 2)
 
 
-def cut_into_parts(n_items, D, R, C):
-    """The library's host rule, restated: are the work items of the last wave cut into parts?
-    (Head dimension 128 with 128-row query blocks runs on pairs of CTAs: half as many slots.)"""
-    ctas = min(torch.cuda.get_device_properties(0).multi_processor_count, 160)
-    if D == 128 and R == 128:
-        ctas //= 2
+def cut_into_parts(n_items, B, H, N, D, R, C):
+    """Are the work items of the last wave cut into parts?  (The slots come from the library.)"""
+    losa = lib()
+    prob = losa.make_problem(torch.empty((B, H, N, D), dtype=torch.bfloat16, device="cuda"), R, C)
+    ctas = losa.losa_work_slots(losa.binding.LOSA_OP_SPARSE_ATTN, prob)
+    assert ctas > 0
     rest = n_items if n_items < ctas else n_items % ctas
     return rest > 0 and ctas // rest >= 2
 
@@ -50,7 +50,7 @@ def cut_into_parts(n_items, D, R, C):
 def test_three_layers_in_one_launch_equal_the_single_calls_bit_for_bit(B, H, N, D, R, C):
     losa = lib()
     L = 3
-    if cut_into_parts(items(B, H, N), D, R, C) or cut_into_parts(L * items(B, H, N), D, R, C):
+    if cut_into_parts(items(B, H, N), B, H, N, D, R, C) or cut_into_parts(L * items(B, H, N), B, H, N, D, R, C):
         pytest.skip("this GPU's SM count cuts the last wave into parts for this shape")
     host, dev = make_layers(L, B, H, N, D, R, C, 300)
     outs = losa.losa_sparse_attn_batched(dev, R, C, out_dtype=torch.float32)
