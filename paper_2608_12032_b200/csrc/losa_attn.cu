@@ -57,6 +57,9 @@ namespace {
 #ifndef LOSA_PAIR_FUSED
 #define LOSA_PAIR_FUSED 1
 #endif
+#ifndef LOSA_PAIR_MASS
+#define LOSA_PAIR_MASS 1
+#endif
 #ifndef LOSA_PAIR_MIN_C
 #define LOSA_PAIR_MIN_C 32
 #endif
@@ -2050,9 +2053,12 @@ int launch_t(const Geometry& g, const void* q, const void* k, const void* v, Par
   // one work item per pair at a time (see losa_attn_pair.cuh); the single-CTA kernels stay the
   // fallback.  (With 32-key blocks the pair kernel was slower than the single-CTA kernel until
   // tiles of consecutive key blocks were copied whole: dense forward 6.3 against 5.9 ms before,
-  // 5.56 against 6.20 ms after.)
+  // 5.56 against 6.20 ms after.)  The mass pass alone runs on pairs only with 32-key blocks (5.65 -> 5.16
+  // ms at the Wan shape; with 64- and 128-key blocks it measured the same or 2 % slower on pairs: the
+  // exponential unit bounds it either way).
   constexpr bool kPairMode = LOSA_USE_PAIR && D == 128 && R == 128 && C_ >= LOSA_PAIR_MIN_C &&
-                             (MODE == kDense || MODE == kSparse || (LOSA_PAIR_FUSED && MODE == kFused));
+                             (MODE == kDense || MODE == kSparse || (LOSA_PAIR_FUSED && MODE == kFused) ||
+                              (LOSA_PAIR_MASS && MODE == kMass && C_ < 64));
   bool pair = false;  // (a device that cannot hold a pair of these CTAs runs the single-CTA kernel)
   CUtensorMap mkh, mk64;
   if constexpr (kPairMode) {
@@ -2169,7 +2175,8 @@ void arm_stalled_launch(uint32_t polls) { g_stall_polls.store(polls); }
 int attn_work_slots(AttnMode mode, const Geometry& g, int sms) {
   const int ctas = sms < kMaxPersistentCtas ? sms : kMaxPersistentCtas;
   const bool pair = LOSA_USE_PAIR && g.D == 128 && g.R == 128 && g.C >= LOSA_PAIR_MIN_C &&
-                    (mode == kDense || mode == kSparse || (LOSA_PAIR_FUSED && mode == kFused)) && sms >= 2;
+                    (mode == kDense || mode == kSparse || (LOSA_PAIR_FUSED && mode == kFused) ||
+                     (LOSA_PAIR_MASS && mode == kMass && g.C < 64)) && sms >= 2;
   return pair ? ctas / 2 : ctas;
 }
 

@@ -139,7 +139,9 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   constexpr uint32_t kIdescQK = ptx::idesc_bf16_f32(256, 128, false, false);
   constexpr uint32_t kIdescPV = ptx::idesc_bf16_f32(256, 128, false, true);
   using Ctl = PairControl;
-  constexpr bool kWantMass = (MODE == kFused);  // the construction step: dense O and the block masses
+  constexpr bool kWantMass = (MODE == kFused || MODE == kMass);  // the block masses (Eq. 1) are wanted
+  // the mass pass alone has no V, no P and no O: its score buffers go back as soon as they are read
+  constexpr bool kHasV = (MODE != kMass);
   static_assert(offsetof(PairControl, tl) % 16 == 0, "the tile list is read with 16-byte loads");
 
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -301,6 +303,7 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                                   s * 64, r0, h, b);
           }
           ++nk;
+          if (!kHasV) continue;
           // V: all 128 keys of the tile, head-dimension columns 64 * rank ... + 63 (one slab)
           const uint32_t vs = nv % kPairNV;
           LOSA_WAIT_RELAXED(&ctl->v_empty[vs], ((nv / kPairNV) & 1) ^ 1);
@@ -357,7 +360,11 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             q_ready = true;
           }
           const uint32_t bsel = nt % 3u;
-          if (nt >= 3u) LOSA_WAIT(&ctl->pv_done[bsel], (nt / 3u - 1u) & 1);
+          if (nt >= 3u) {
+            // (mass pass: the softmax warps of both CTAs hand the buffer back once it is in registers)
+            if (kHasV) LOSA_WAIT(&ctl->pv_done[bsel], (nt / 3u - 1u) & 1);
+            else LOSA_WAIT(&ctl->p_ready[bsel], (nt / 3u - 1u) & 1);
+          }
           ptx::tc_fence_after_sync();
           if (leader) {
             const uint32_t kd0 = k_lo + ks * (kPairStage >> 4);
@@ -395,6 +402,7 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             ent = grp[0];
             break;
           }
+          if (!kHasV) continue;  // (mass pass: this warp only hands the list's chunks back)
           const uint32_t vs = nt % kPairNV;
           LOSA_WAIT(&ctl->v_full[vs], (nt / kPairNV) & 1);
           const uint32_t bsel = nt % 3u;
@@ -606,6 +614,13 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 if ((c % kBW) >= hv[c / kBW]) sr[c] = 0xff800000u;
             }
           }
+          if (!kHasV) {
+            // mass pass: the scores are in registers and nothing is packed over them
+            ptx::tmem_wait_ld();
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(p_ready0 + 8u * bsel);
+          }
           // key blocks the row's query block does not list get -inf as the addend of the scaling FMA
           const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
           float2 nm2[kHB];
@@ -622,7 +637,7 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           for (int i = 0; i < kHB; ++i) eacc[i] = make_float2(0.f, 0.f);
 #pragma unroll
           for (int c = 0; c < 64; c += 4) {
-            if (whole && c == 32) ptx::tmem_wait_ld();
+            if (kHasV && whole && c == 32) ptx::tmem_wait_ld();
             float2 x0 = ptx::fma2(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2,
                                   nm2[c / kBW]);
             float2 x1 = ptx::fma2(make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2,
@@ -633,17 +648,23 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             x0.y = ptx::ex2_approx(x0.y);
             x1.x = ptx::ex2_approx(x1.x);
             x1.y = ptx::ex2_approx(x1.y);
-            const uint32_t u0 = ptx::pack_bf16x2(x0.x, x0.y), u1 = ptx::pack_bf16x2(x1.x, x1.y);
-            sr[c >> 1] = u0;
-            sr[(c >> 1) + 1] = u1;
-            ptx::add_bf16x2(racc[0], u0);
-            ptx::add_bf16x2(racc[1], u1);
+            if (kHasV) {
+              const uint32_t u0 = ptx::pack_bf16x2(x0.x, x0.y), u1 = ptx::pack_bf16x2(x1.x, x1.y);
+              sr[c >> 1] = u0;
+              sr[(c >> 1) + 1] = u1;
+              ptx::add_bf16x2(racc[0], u0);
+              ptx::add_bf16x2(racc[1], u1);
+            }
             if (kWantMass) eacc[c / kBW] = ptx::add2(eacc[c / kBW], ptx::add2(x0, x1));
           }
-          const float tsum = (racc[0].x + racc[0].y) + (racc[1].x + racc[1].y);
+          float tsum = (racc[0].x + racc[0].y) + (racc[1].x + racc[1].y);
+          if (!kHasV) {
+#pragma unroll
+            for (int i = 0; i < kHB; ++i) tsum += eacc[i].x + eacc[i].y;
+          }
           ovf = ovf || __any_sync(0xffffffffu, !(tsum <= kSplitSafeSum));
           l += tsum;
-          ptx::tmem_st32(tS, &sr[0]);
+          if (kHasV) ptx::tmem_st32(tS, &sr[0]);
           if (kWantMass) {
 #pragma unroll
             for (int i = 0; i < kHB; ++i) {
@@ -656,19 +677,28 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
         } else {
           // this half of the row lists none of the tile's keys: P = 0
-          uint32_t z[32];
+          if (kHasV) {
+            uint32_t z[32];
 #pragma unroll
-          for (int c = 0; c < 32; ++c) z[c] = 0u;
-          ptx::tmem_st32(tS, z);
+            for (int c = 0; c < 32; ++c) z[c] = 0u;
+            ptx::tmem_st32(tS, z);
+          } else {
+            // mass pass: the buffer goes back untouched
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(p_ready0 + 8u * bsel);
+          }
           // (a key block that fills the tile but ends before this half: its entry of the table is 0)
           if (kWantMass && kG == 1 && member &&
               LOSA_IN_RANGE(((int64_t)(grp[0] & 0xffffu) * 2 + half) * 128 + row, p.cap_table_floats))
             tabf[((int64_t)(grp[0] & 0xffffu) * 2 + half) * 128] = 0.f;
         }
-        ptx::tmem_wait_st();
-        ptx::tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive_cluster(p_ready0 + 8u * bsel);
+        if (kHasV) {
+          ptx::tmem_wait_st();
+          ptx::tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive_cluster(p_ready0 + 8u * bsel);
+        }
       }
 
       // ---- end of the item
@@ -700,7 +730,7 @@ losa_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       LOSA_WAIT(&ctl->item_bar, nitem & 1);
       ++nitem;
       l = (xset[row] + xset[128 + row]) + (xset[256 + row] + xset[384 + row]);
-      {
+      if (kHasV) {
         // every thread writes out a quarter (32 columns) of its row of O
         const bool valid = (T < p.nQt) && grow < p.N;
         const float inv = (l > 0.f) ? 1.f / l : 0.f;
